@@ -13,9 +13,9 @@ Models"):
                            M_t), the refresh paragraph of Sec. 3.3, the
                            Prefill / PD paragraph, Sec. 3.4 (Greedy + window).
 * ``concat_reorder_maps``  Appendix A: the two physical orders and the map I'.
-* ``LiteralCache.step``    Algorithm 1, line by line (gather rows, reorder the
-                           positional encoding, transformer on the active rows,
-                           Concat, Reorder, attention, scatter back).
+* ``LiteralCache.step``    Sec. 3.3 / Appendix A / Algorithm 1: the cache as physically
+                           ordered arrays (cached rows, then fresh rows), narrowed
+                           through index maps, concatenated for the attention of Eq. 4.
 * ``SlotCache.step``       the same step written with position-addressed
                            slots; ``tests`` check literal == slots.
 * ``select_unmask``        Sec. 3.1, "keeping the most confident ones".
@@ -240,7 +240,7 @@ def vanilla_forward(model: Model, W: Dict, x: np.ndarray, rnd=_identity) -> np.n
 
 
 def _scatter_logits(fw: "_Forward", h: np.ndarray, A: np.ndarray, logit_rows, L: int) -> "SparseLogits":
-    """Logits of the wanted rows, addressed by ORIGINAL position (Alg. 1 l.7)."""
+    """Logits of the wanted rows, addressed by ORIGINAL position (the scatter that ends Algorithm 1)."""
     if logit_rows is None:
         sel = np.arange(len(A))
     else:
@@ -285,15 +285,20 @@ class SparseLogits:
 
 
 class LiteralCache:
-    """Algorithm 1 written out.  Per layer the cache is a pair of arrays whose
-    rows are in PHYSICAL order ``self.order`` (cached rows on the left, the
-    rows computed in the last step on the right); nothing is addressed by
-    position except through ``self.order``."""
+    """The cache as Sec. 3.3 and Appendix A describe it: per layer a pair of
+    arrays whose rows sit in a PHYSICAL order (``self.order`` lists the position
+    each physical row belongs to), cached rows first, the rows computed in the
+    last evaluation behind them.  Nothing is addressed by position: a step
+    first narrows the arrays to the rows it will serve from the cache, appends
+    the freshly computed rows (Eq. 4: K of the cached set next to K of the
+    active set), attends over the concatenation, and finally narrows again to
+    what the following step may reuse.  Narrowing goes through an index map
+    into the current physical order (the map I' of Appendix A)."""
 
     def __init__(self, model: Model, W: Dict, L: int, rnd=_identity):
         self.fw = _Forward(model, W, rnd)
         self.m, self.L = model, L
-        self.order: List[int] = []                 # positions held, physical order
+        self.order: List[int] = []                 # position of each physical row
         self.K: List[Optional[np.ndarray]] = [None] * model.n_layers
         self.V: List[Optional[np.ndarray]] = [None] * model.n_layers
         self.written_step = np.zeros(L, dtype=np.int64)
@@ -308,55 +313,49 @@ class LiteralCache:
         self.order = list(range(P))
         self.written_step[:P] = self.t + 1
 
-    def drop_except(self, keep: Sequence[int]):
-        """Reorder (Alg. 1 line 5): keep only the positions of ``keep``, in
-        that order, using the index map I' into the current physical order."""
-        where = {p: j for j, p in enumerate(self.order)}
-        idx = np.array([where[p] for p in keep], dtype=np.int64)
+    def narrow_to(self, keep: Sequence[int]):
+        """Physical rows become exactly the positions ``keep``, in that order
+        (gather through the index map into the present order)."""
+        present = {p: j for j, p in enumerate(self.order)}
+        imap = np.array([present[p] for p in keep], dtype=np.int64)
         for l in range(self.m.n_layers):
             if self.K[l] is not None:
-                self.K[l] = self.K[l][idx]
-                self.V[l] = self.V[l][idx]
+                self.K[l], self.V[l] = self.K[l][imap], self.V[l][imap]
         self.order = list(keep)
 
     def step(self, x: np.ndarray, A: np.ndarray, keep_after: Optional[Sequence[int]] = None,
              logit_rows: Optional[Sequence[int]] = None):
-        """One model evaluation with active rows A (ascending positions).
-        Returns logits for the rows of A, as an [L, V] array that is NaN
-        outside A (Alg. 1 line 7: scatter back to the original positions).
-        keep_after: positions to keep as the next step's cache (Alg. 1 l.5);
-        None keeps every position.  logit_rows: positions (a subset of A)
-        whose logits are wanted; the head is row-wise, so leaving the other
-        rows out changes nothing for these (None = all of A, as Alg. 1)."""
+        """One model evaluation in which the rows A (ascending positions) are
+        recomputed and every other position is served from the cache.
+        keep_after: the positions the following step will serve from the cache,
+        when already known (None keeps every row).  logit_rows: positions (a
+        subset of A) whose logits are wanted; the head is row-wise, so leaving
+        the other rows out changes nothing for these (None = all of A).
+        Returns the logits addressed by ORIGINAL position."""
         self.t += 1
         m, L = self.m, self.L
         A = np.asarray(A, dtype=np.int64)
-        Aset = set(A.tolist())
-        cached = [p for p in range(L) if p not in Aset]           # I \ A
-        held = set(self.order)
-        missing = [p for p in cached if p not in held]
-        if missing:
-            raise KeyError(f"step {self.t}: cached K/V missing for positions {missing[:8]}")
-        # gather the cached rows to the left (index map into the held order)
-        self.drop_except(cached)
-        xp = x[A]                                                 # line 1
-        pe = np.concatenate([np.array(cached, dtype=np.int64), A])  # line 2
-        pe_active = pe[len(cached):]
-        h = self.fw.embed(xp)
+        recomputed = set(A.tolist())
+        stable = [p for p in range(L) if p not in recomputed]     # served from the cache this step
+        absent = sorted(set(stable) - set(self.order))
+        if absent:
+            raise KeyError(f"step {self.t}: cached K/V missing for positions {absent[:8]}")
+        self.narrow_to(stable)
+        h = self.fw.embed(x[A])
         for l in range(m.n_layers):
-            q, k, v = self.fw.qkv(l, h, pe_active)                # line 3
-            if len(cached):
-                Kall = np.concatenate([self.K[l], k], axis=0)     # line 4
-                Vall = np.concatenate([self.V[l], v], axis=0)
+            # rotary phases follow the rows' original positions, whatever their physical place
+            q, k_new, v_new = self.fw.qkv(l, h, A)
+            if stable:
+                self.K[l] = np.concatenate([self.K[l], k_new], axis=0)
+                self.V[l] = np.concatenate([self.V[l], v_new], axis=0)
             else:
-                Kall, Vall = k, v
-            self.K[l], self.V[l] = Kall, Vall
-            h = self.fw.after_attention(l, h, attention(q, Kall, Vall))  # line 6
-        self.order = cached + A.tolist()
+                self.K[l], self.V[l] = k_new, v_new
+            h = self.fw.after_attention(l, h, attention(q, self.K[l], self.V[l]))
+        self.order = stable + A.tolist()
         self.written_step[A] = self.t
         if keep_after is not None:
-            self.drop_except(list(keep_after))                    # line 5
-        return _scatter_logits(self.fw, h, A, logit_rows, L)      # line 7
+            self.narrow_to(list(keep_after))
+        return _scatter_logits(self.fw, h, A, logit_rows, L)
 
 
 class SlotCache:
@@ -513,7 +512,7 @@ class Sampler:
         if pol.shift:
             assert len(H) == 0 or H.min() >= 1, "a shifted head cannot predict position 0"
             A = np.union1d(A, src).astype(np.int64)
-        # what the next step will read from the cache, when already known (Alg. 1 l.5)
+        # what the next step will read from the cache, when already known (Algorithm 1's Reorder)
         keep_after = None
         if self.form == "literal" and pol.kind in (POLICY_DECODE, POLICY_PD) and pol.delay == 1:
             keep_after = [p for p in range(L) if not M[p]]      # next active set is M_t

@@ -5,7 +5,8 @@
 // row, query head of the KV head's group) pair, so GQA groups share the K/V
 // tiles.  Q, K and V tiles are TMA-loaded (128-byte swizzle); K/V come straight
 // from the position-addressed slot cache, BKV slots per iteration, double
-// buffered.  Two shapes of the same kernel: <128 slots, two softmax warpgroups>,
+// buffered; the K/V maps are 3-D [head][slot][head_dim], so a tile that reaches past the last slot is
+// zero-filled and never sees a neighbouring head's or layer's memory.  Two shapes of the same kernel: <128 slots, two softmax warpgroups>,
 // one CTA per SM, for launches that do not fill the GPU twice (shortest latency
 // per CTA), and <64 slots, one warpgroup>, two CTAs per SM, for large launches:
 // within one CTA the tensor pipe, the special-function unit and the tensor-memory
@@ -44,11 +45,10 @@ constexpr long long ATC_WAIT_CYCLES = 4000000000LL;
 struct AttnTcParams {
   void* o;                  // [R, H_q, 128] 16-bit
   const int32_t* row_off;   // [B+1]
-  int seq_len, n_q_heads, n_kv_heads;
-  int kv_stride;       // slots per head in memory; the first seq_len of them are attended
+  int seq_len, n_q_heads, n_kv_heads;   // seq_len = attended slots = the slot extent of the K/V tensor maps
   int group;                // query heads per KV head
   int rows_q;               // query rows per tile = 128 / group
-  long long kv_row0;        // first row of this layer inside the K/V tensor maps
+  int kv_head0;             // first KV head of this layer inside the K/V tensor maps
   float scale_log2;
   int bf16;                 // 1: bf16 operands, 0: fp16
   int* status;
@@ -176,7 +176,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   const int q0 = blockIdx.x * p.rows_q;
   const bool active = q0 < n_a && !*abort_flag;   // uniform over the CTA
   const int n_iter = active ? (p.seq_len + BKV - 1) / BKV : 0;
-  const long long kv_row = p.kv_row0 + (static_cast<long long>(b) * p.n_kv_heads + hk) * p.kv_stride;
+  const int kv_head = p.kv_head0 + b * p.n_kv_heads + hk;    // index into the maps' outermost dimension
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA
@@ -187,15 +187,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       for (int j = 0; j < n_iter; ++j) {
         const int s = j & 1;
         const uint32_t base = sKV + s * 4 * KVT;
-        const int row = static_cast<int>(kv_row + static_cast<long long>(j) * BKV);
+        const int row = j * BKV;      // slots past seq_len are zero-filled by the copy (3-D map)
         if (!mbar_wait_bounded(smem_u32(&k_empty[s]), ((j >> 1) & 1) ^ 1, abort_flag, ATC_WAIT_CYCLES)) break;
         const uint32_t kf = smem_u32(&k_full[s]);
         mbar_expect_tx(kf, 2 * KVT);
-        for (int half = 0; half < 2; ++half) tma_load_2d(base + half * KVT, &tm_k, kf, half * 64, row);
+        for (int half = 0; half < 2; ++half) tma_load_3d(base + half * KVT, &tm_k, kf, half * 64, row, kv_head);
         if (!mbar_wait_bounded(smem_u32(&v_empty[s]), ((j >> 1) & 1) ^ 1, abort_flag, ATC_WAIT_CYCLES)) break;
         const uint32_t vf = smem_u32(&v_full[s]);
         mbar_expect_tx(vf, 2 * KVT);
-        for (int half = 0; half < 2; ++half) tma_load_2d(base + (2 + half) * KVT, &tm_v, vf, half * 64, row);
+        for (int half = 0; half < 2; ++half) tma_load_3d(base + (2 + half) * KVT, &tm_v, vf, half * 64, row, kv_head);
       }
     }
   } else if (warp == 1) {

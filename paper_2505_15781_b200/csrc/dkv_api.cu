@@ -9,7 +9,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <unordered_set>
 #include <vector>
 
 #include "../../include/dkv.h"
@@ -132,8 +134,11 @@ struct AttnMaps {
   CUtensorMap k64, v64;     // K/V boxes of 64 slots (two CTAs per SM)
   int group, rows_q;
 };
+// K and V slots as a 3-D tensor [KV heads of all layers and sequences][kv_len slots][128]: a slot tile that
+// reaches past kv_len is zero-filled by the copy engine instead of running into the next head's (or the
+// next layer's, possibly unwritten) slots.  kv_stride = slots per head in memory (>= kv_len).
 int make_attn_maps(AttnMaps* am, const void* q, long long q_rows, const void* k_slots, const void* v_slots,
-                   long long kv_rows, int hq, int hkv, bool fp16) {
+                   long long kv_heads_total, int kv_len, int kv_stride, int hq, int hkv, bool fp16) {
   am->group = hq / hkv;
   am->rows_q = ATC_M / am->group;
   if (am->rows_q < 1) return DKV_E_UNSUPPORTED;
@@ -141,19 +146,22 @@ int make_attn_maps(AttnMaps* am, const void* q, long long q_rows, const void* k_
   cuuint64_t qs[2] = {static_cast<cuuint64_t>(ATC_DH) * 2, static_cast<cuuint64_t>(hq) * ATC_DH * 2};
   cuuint32_t qb[3] = {64, static_cast<cuuint32_t>(am->group), static_cast<cuuint32_t>(am->rows_q)};
   int rc = make_tmap_nd(&am->q, q, 3, qd, qs, qb, fp16);
-  cuuint64_t kd[2] = {static_cast<cuuint64_t>(ATC_DH), static_cast<cuuint64_t>(kv_rows)};
-  cuuint64_t ks[1] = {static_cast<cuuint64_t>(ATC_DH) * 2};
-  cuuint32_t kb[2] = {64, ATC_BKV};
-  if (!rc) rc = make_tmap_nd(&am->k, k_slots, 2, kd, ks, kb, fp16);
-  if (!rc) rc = make_tmap_nd(&am->v, v_slots, 2, kd, ks, kb, fp16);
-  cuuint32_t kb64[2] = {64, 64};
-  if (!rc) rc = make_tmap_nd(&am->k64, k_slots, 2, kd, ks, kb64, fp16);
-  if (!rc) rc = make_tmap_nd(&am->v64, v_slots, 2, kd, ks, kb64, fp16);
+  cuuint64_t kd[3] = {static_cast<cuuint64_t>(ATC_DH), static_cast<cuuint64_t>(kv_len),
+                      static_cast<cuuint64_t>(kv_heads_total)};
+  cuuint64_t ks[2] = {static_cast<cuuint64_t>(ATC_DH) * 2, static_cast<cuuint64_t>(kv_stride) * ATC_DH * 2};
+  cuuint32_t kb[3] = {64, ATC_BKV, 1};
+  if (!rc) rc = make_tmap_nd(&am->k, k_slots, 3, kd, ks, kb, fp16);
+  if (!rc) rc = make_tmap_nd(&am->v, v_slots, 3, kd, ks, kb, fp16);
+  cuuint32_t kb64[3] = {64, 64, 1};
+  if (!rc) rc = make_tmap_nd(&am->k64, k_slots, 3, kd, ks, kb64, fp16);
+  if (!rc) rc = make_tmap_nd(&am->v64, v_slots, 3, kd, ks, kb64, fp16);
   return rc;
 }
 
-int attention_tc(const AttnMaps& am, void* o, const int32_t* row_off, int batch, int rows_bound, int seq_len, int hq,
-                 int hkv, long long kv_row0, bool bf16, int* status, cudaStream_t st, int kv_stride = 0) {
+// kv_len: the slots every query attends = the slot extent of am's K/V maps; kv_head0: first KV head of
+// this layer inside the maps.
+int attention_tc(const AttnMaps& am, void* o, const int32_t* row_off, int batch, int rows_bound, int kv_len, int hq,
+                 int hkv, int kv_head0, bool bf16, int* status, cudaStream_t st) {
   static PerDeviceOnce attr_once;
   if (attr_once.need()) {
     if (cudaFuncSetAttribute(k_attn_tc<128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_tc_smem<128, 2>()) !=
@@ -162,17 +170,15 @@ int attention_tc(const AttnMaps& am, void* o, const int32_t* row_off, int batch,
             cudaSuccess)
       return DKV_E_CUDA;
   }
-  static const int env_shape = env_int("DKV_ATTN_SHAPE", 0);   // 1: always 128 slots, 2: always 64 slots
   AttnTcParams p;
   p.o = o;
   p.row_off = row_off;
-  p.seq_len = seq_len;
-  p.kv_stride = kv_stride > 0 ? kv_stride : seq_len;
+  p.seq_len = kv_len;
   p.n_q_heads = hq;
   p.n_kv_heads = hkv;
   p.group = am.group;
   p.rows_q = am.rows_q;
-  p.kv_row0 = kv_row0;
+  p.kv_head0 = kv_head0;
   p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(ATC_DH));
   p.bf16 = bf16 ? 1 : 0;
   p.status = status;
@@ -180,8 +186,7 @@ int attention_tc(const AttnMaps& am, void* o, const int32_t* row_off, int batch,
   // Two resident CTAs per SM keep the units busy; with at most one CTA per SM to hand out, the
   // 128-slot shape has half the iterations and the shorter latency.
   const long long ctas = static_cast<long long>(grid.x) * grid.y * grid.z;
-  const bool small_tiles = env_shape ? env_shape == 2 : ctas > 148;
-  if (small_tiles)
+  if (ctas > 148)
     launch_k((k_attn_tc<64, 1>), grid, 192, attn_tc_smem<64, 1>(), st, am.q, am.k64, am.v64, p);
   else
     launch_k((k_attn_tc<128, 2>), grid, 320, attn_tc_smem<128, 2>(), st, am.q, am.k, am.v, p);
@@ -339,13 +344,15 @@ struct dkv_cache {
   Arena ar;
   CUtensorMap xmaps[XB_COUNT][N_BOX];
   CUtensorMap xmaps_half[N_BOX];   // the normalised rows (XB_XN) in boxes of half the rows, for the CTA-pair GEMM
-  AttnMaps attn_maps;            // tcgen05 attention (head_dim 128, 16-bit modes)
+  AttnMaps attn_maps;            // tcgen05 attention (head_dim 128, 16-bit modes): all seq_len slots attended
+  AttnMaps attn_maps_prompt;     // the same buffers with the slot extent cut at the prompt (isolated prefill pass)
   bool attn_tc;
   int step;              // steps run so far
   int last_refresh;      // step number of the last full / generation-only step
   int pending_refresh;   // -1 none, else DKV_REFRESH_*
   int prev_rows_bound;   // bound on #M_{t-1} per sequence
   bool have_dprev;
+  int prev_k;            // k of the step that stored D_{t-1}
   cudaStream_t last_stream;
   dkv_stats stats;
   bool profiling;
@@ -355,6 +362,30 @@ struct dkv_cache {
 };
 
 namespace {
+
+// Live handles: every entry point checks its handle against these sets, so that a destroyed,
+// never-created or foreign pointer yields DKV_E_STATE instead of undefined behaviour.
+std::mutex g_live_mu;
+std::unordered_set<const void*> g_live_models, g_live_caches;
+bool live_model(const dkv_model* m) {
+  std::lock_guard<std::mutex> lk(g_live_mu);
+  return g_live_models.count(m) != 0;
+}
+bool live_cache(const dkv_cache* c) {
+  std::lock_guard<std::mutex> lk(g_live_mu);
+  return g_live_caches.count(c) != 0 && g_live_models.count(c->model) != 0;
+}
+void set_live(std::unordered_set<const void*>& set, const void* h, bool on) {
+  std::lock_guard<std::mutex> lk(g_live_mu);
+  if (on) set.insert(h);
+  else set.erase(h);
+}
+// NULL -> INVALID_ARG, not a live handle (or its model was destroyed) -> STATE
+#define DKV_CHECK_CACHE(c)             \
+  do {                                 \
+    if (!(c)) return DKV_E_INVALID_ARG; \
+    if (!live_cache(c)) return DKV_E_STATE; \
+  } while (0)
 
 // --------------------------------------------------------------- profiling
 void prof_flush(dkv_cache* c) {
@@ -740,8 +771,8 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       const double by = 2.0 * dm.B * dm.L * dkv * es + 2.0 * R * dq * es;
       Launch lk(c, st, PC_ATTN, by, fl);
       if (bf16 && c->attn_tc)
-        rc = attention_tc(c->attn_maps, a.ao, a.row_off, dm.B, plan.na_bound, kv_count, md.n_q_heads, md.n_kv_heads,
-                          static_cast<long long>(l) * dm.B * md.n_kv_heads * dm.L, x_bf16, a.status, st, dm.L);
+        rc = attention_tc(kv_count < dm.L ? c->attn_maps_prompt : c->attn_maps, a.ao, a.row_off, dm.B, plan.na_bound,
+                          kv_count, md.n_q_heads, md.n_kv_heads, l * dm.B * md.n_kv_heads, x_bf16, a.status, st);
       else
         rc = attention_any(static_cast<const T*>(a.qb), static_cast<const T*>(ks), static_cast<const T*>(vs),
                            static_cast<T*>(a.ao), a.row_off, dm.B, plan.na_bound, kv_count, md.n_q_heads, md.n_kv_heads,
@@ -893,6 +924,8 @@ int do_step(dkv_cache* c, const int32_t* tokens, const uint8_t* masked, const in
   if (k < 1 || k > dm.kmax) return DKV_E_SHAPE;
   if (cand_lo < 0 || cand_hi > dm.L || cand_lo > cand_hi) return DKV_E_SHAPE;
   if (pol.kind == DKV_POLICY_GREEDY && !next_pos) return DKV_E_INVALID_ARG;
+  // D_{t-1} was stored as [batch, k] with the previous step's k: the window rule reads it with the same k
+  if (pol.kind == DKV_POLICY_GREEDY && c->have_dprev && k != c->prev_k) return DKV_E_SHAPE;
   if (pol.shift && cand_lo < 1) return DKV_E_SHAPE;   // position 0 has no row to its left
   StepPlan plan = plan_step(c, k, cand_lo, cand_hi, rows_bound);
   if (plan.nh_bound > dm.hmax) return DKV_E_SHAPE;
@@ -966,6 +999,7 @@ int do_step(dkv_cache* c, const int32_t* tokens, const uint8_t* masked, const in
   c->pending_refresh = -1;
   c->prev_rows_bound = rows_bound < 0 ? dm.L : std::min(rows_bound, dm.L);
   c->have_dprev = next_pos != nullptr;
+  c->prev_k = k;
   c->last_stream = st;
   c->stats.steps += 1;
   if (plan.refresh) c->stats.refresh_steps += 1;
@@ -1085,17 +1119,21 @@ int dkv_model_create(const dkv_model_desc* desc, const dkv_weights* w, void* are
       return rc;
     }
   }
+  set_live(g_live_models, m, true);
   *out = m;
   return DKV_OK;
 }
 
 int dkv_model_destroy(dkv_model* m) {
+  if (!m) return DKV_OK;
+  if (!live_model(m)) return DKV_E_STATE;
+  set_live(g_live_models, m, false);
   delete m;
   return DKV_OK;
 }
 
 size_t dkv_cache_bytes(const dkv_model* m, int batch, int seq_len, const dkv_policy* policy) {
-  if (!m || batch < 1 || seq_len < 1) return 0;
+  if (!m || !live_model(m) || batch < 1 || seq_len < 1) return 0;
   Dims d = make_dims(m, batch, seq_len, 0, policy);
   Arena a;
   carve(m, d, nullptr, &a);
@@ -1105,6 +1143,7 @@ size_t dkv_cache_bytes(const dkv_model* m, int batch, int seq_len, const dkv_pol
 int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, const dkv_policy* policy, void* arena,
                    size_t arena_bytes, void* stream, dkv_cache** out) {
   if (!m || !policy || !arena || !out) return DKV_E_INVALID_ARG;
+  if (!live_model(m)) return DKV_E_STATE;
   if (batch < 1 || seq_len < 1 || prompt_len < 0 || prompt_len > seq_len) return DKV_E_SHAPE;
   if (policy->kind < DKV_POLICY_NONE || policy->kind > DKV_POLICY_GREEDY) return DKV_E_INVALID_ARG;
   if (policy->refresh_interval < 0 || policy->window < 0) return DKV_E_INVALID_ARG;
@@ -1140,9 +1179,13 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
     static const int env_attn_tc = env_int("DKV_ATTN_TC", 1);
     c->attn_tc = false;
     if (!rc && md.head_dim == ATC_DH && env_attn_tc && md.n_q_heads / md.n_kv_heads <= ATC_M) {
-      const long long kv_rows = static_cast<long long>(md.n_layers) * batch * md.n_kv_heads * seq_len;
-      rc = make_attn_maps(&c->attn_maps, a.qb, c->dims.r_cap, a.k_slots, a.v_slots, kv_rows, md.n_q_heads,
-                          md.n_kv_heads, md.act_dtype == DKV_F16);
+      const long long kv_heads = static_cast<long long>(md.n_layers) * batch * md.n_kv_heads;
+      const bool h16 = md.act_dtype == DKV_F16;
+      rc = make_attn_maps(&c->attn_maps, a.qb, c->dims.r_cap, a.k_slots, a.v_slots, kv_heads, seq_len, seq_len,
+                          md.n_q_heads, md.n_kv_heads, h16);
+      if (!rc && policy->isolated_prefill && prompt_len > 0 && prompt_len < seq_len)
+        rc = make_attn_maps(&c->attn_maps_prompt, a.qb, c->dims.r_cap, a.k_slots, a.v_slots, kv_heads, prompt_len,
+                            seq_len, md.n_q_heads, md.n_kv_heads, h16);
       c->attn_tc = rc == DKV_OK;
     }
     if (rc) {
@@ -1162,13 +1205,6 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   cudaMemsetAsync(a.ao, 0, c->dims.r_cap * m->d_q * m->asize, st);
   cudaMemsetAsync(a.ub, 0, c->dims.r_cap * md.d_ffn * m->asize, st);
   cudaMemsetAsync(a.xh, 0, c->dims.h_cap * md.d_model * m->asize, st);
-  if (policy->isolated_prefill) {
-    // the prefill pass loads slot tiles that reach past the prompt; masked scores times an
-    // unwritten value must be 0, not NaN
-    const size_t slots = static_cast<size_t>(md.n_layers) * batch * md.n_kv_heads * seq_len * md.head_dim * m->asize;
-    cudaMemsetAsync(a.k_slots, 0, slots, st);
-    cudaMemsetAsync(a.v_slots, 0, slots, st);
-  }
   {
     const int half = md.head_dim / 2;
     const int n = seq_len * half;
@@ -1183,6 +1219,7 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   c->pending_refresh = -1;
   c->prev_rows_bound = seq_len;
   c->have_dprev = false;
+  c->prev_k = 0;
   c->last_stream = st;
   memset(&c->stats, 0, sizeof(c->stats));
   c->stats.cache_bytes = 2LL * md.n_layers * batch * md.n_kv_heads * seq_len * md.head_dim * m->asize;
@@ -1190,12 +1227,18 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   c->ev_used = 0;
   memset(c->prof, 0, sizeof(c->prof));
   for (int i = 0; i < PC_COUNT; ++i) strncpy(c->prof[i].name, PROF_NAMES[i], sizeof(c->prof[i].name) - 1);
+  set_live(g_live_caches, c, true);
   *out = c;
   return DKV_OK;
 }
 
 int dkv_cache_destroy(dkv_cache* c) {
   if (!c) return DKV_OK;
+  {
+    std::lock_guard<std::mutex> lk(g_live_mu);
+    if (!g_live_caches.count(c)) return DKV_E_STATE;
+    g_live_caches.erase(c);
+  }
   for (ProfEvent& e : c->events) {
     cudaEventDestroy(e.a);
     cudaEventDestroy(e.b);
@@ -1207,12 +1250,13 @@ int dkv_cache_destroy(dkv_cache* c) {
 int dkv_step(dkv_cache* c, const int32_t* tokens, const uint8_t* masked, const int32_t* next_pos, int k, int cand_lo,
              int cand_hi, int rows_bound, float* conf, int32_t* pred, float* logits_dbg, void* stream) {
   if (!c || !tokens || !masked || !conf || !pred) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   return do_step(c, tokens, masked, next_pos, k, cand_lo, cand_hi, rows_bound, conf, pred, logits_dbg,
                  static_cast<cudaStream_t>(stream));
 }
 
 int dkv_refresh(dkv_cache* c, int scope) {
-  if (!c) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   if (scope != DKV_REFRESH_ALL && scope != DKV_REFRESH_DECODED_ONLY) return DKV_E_INVALID_ARG;
   c->pending_refresh = scope;
   return DKV_OK;
@@ -1230,6 +1274,7 @@ int dkv_select_unmask(const float* conf, const int32_t* pred, int batch, int seq
 int dkv_step_host(dkv_cache* c, int32_t* tokens_host, uint8_t* masked_host, const int32_t* next_pos_host, int k,
                   int cand_lo, int cand_hi, int rows_bound, int32_t* chosen_host, void* stream) {
   if (!c || !tokens_host || !masked_host) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Arena& a = c->ar;
   const Dims& dm = c->dims;
@@ -1260,6 +1305,7 @@ int dkv_step_host(dkv_cache* c, int32_t* tokens_host, uint8_t* masked_host, cons
 int dkv_generate(dkv_cache* c, int32_t* tokens, uint8_t* masked, const int32_t* order_dev, int k, int block_len,
                  int n_steps, int32_t* chosen_dev, void* stream) {
   if (!c || !tokens || !masked) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   const Dims& dm = c->dims;
   Arena& a = c->ar;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1287,6 +1333,7 @@ int dkv_generate(dkv_cache* c, int32_t* tokens, uint8_t* masked, const int32_t* 
 
 int dkv_get_stats(const dkv_cache* c, dkv_stats* out) {
   if (!c || !out) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   *out = c->stats;
   // the exact number of active rows is counted on the device by the compaction kernel
   unsigned long long act = 0;
@@ -1300,13 +1347,14 @@ int dkv_get_stats(const dkv_cache* c, dkv_stats* out) {
 
 int dkv_get_provenance(const dkv_cache* c, int32_t* written_step, void* stream) {
   if (!c || !written_step) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   cudaError_t e = cudaMemcpyAsync(written_step, c->ar.written_step, static_cast<size_t>(c->dims.B) * c->dims.L * 4,
                                   cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? DKV_OK : DKV_E_CUDA;
 }
 
 int dkv_get_index_maps(const dkv_cache* c, int32_t* act_idx, int32_t* row_off, int32_t* inv, void* stream) {
-  if (!c) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t BL = static_cast<size_t>(c->dims.B) * c->dims.L;
   if (act_idx) cudaMemcpyAsync(act_idx, c->ar.act_idx, BL * 4, cudaMemcpyDeviceToDevice, st);
@@ -1316,7 +1364,7 @@ int dkv_get_index_maps(const dkv_cache* c, int32_t* act_idx, int32_t* row_off, i
 }
 
 int dkv_status(dkv_cache* c, int32_t* word) {
-  if (!c) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   int w = 0;
   if (cudaStreamSynchronize(c->last_stream) != cudaSuccess) return DKV_E_CUDA;
   if (cudaMemcpy(&w, c->ar.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return DKV_E_CUDA;
@@ -1325,7 +1373,8 @@ int dkv_status(dkv_cache* c, int32_t* word) {
 }
 
 int dkv_cache_slots(const dkv_cache* c, int layer, void** k_slots, void** v_slots) {
-  if (!c || layer < 0 || layer >= c->model->desc.n_layers) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
+  if (layer < 0 || layer >= c->model->desc.n_layers) return DKV_E_INVALID_ARG;
   const dkv_model_desc& md = c->model->desc;
   const size_t per = static_cast<size_t>(c->dims.B) * md.n_kv_heads * c->dims.L * md.head_dim * c->model->asize;
   if (k_slots) *k_slots = static_cast<uint8_t*>(c->ar.k_slots) + layer * per;
@@ -1334,7 +1383,7 @@ int dkv_cache_slots(const dkv_cache* c, int layer, void** k_slots, void** v_slot
 }
 
 int dkv_profile_enable(dkv_cache* c, int on) {
-  if (!c) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   if (!on && c->profiling) prof_flush(c);
   c->profiling = on != 0;
   return DKV_OK;
@@ -1342,6 +1391,7 @@ int dkv_profile_enable(dkv_cache* c, int on) {
 
 int dkv_profile_read(dkv_cache* c, dkv_profile_entry* out, int* n) {
   if (!c || !out || !n) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
   prof_flush(c);
   const int cnt = std::min<int>(PC_COUNT, DKV_PROF_CLASSES);
   for (int i = 0; i < cnt; ++i) out[i] = c->prof[i];
@@ -1389,8 +1439,9 @@ int dkv_op_gemm(const void* x, const void* w, float* out, int rows, int n, int k
   rc = gemm_tc(tw, tx, n, k, rows, nullptr, static_cast<float*>(workspace), part_rows, splits, nullptr, dtype == DKV_BF16,
                st, &s, &stride, /*w_static=*/false);
   if (rc || !out) return rc;   // out == NULL: the split-K partials stay in the workspace
-  launch_k(k_reduce_partials, std::min(4 * NUM_SMS, ceil_div(rows * n, 256)), 256, 0, st, 
-      static_cast<const float*>(workspace), s, stride, rows, nullptr, n, out);
+  const long long elems = static_cast<long long>(rows) * n;
+  launch_k(k_reduce_partials, static_cast<int>(std::min<long long>(4 * NUM_SMS, (elems + 255) / 256)), 256, 0, st,
+           static_cast<const float*>(workspace), s, stride, rows, nullptr, n, out);
   return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
 }
 
@@ -1406,8 +1457,8 @@ int dkv_op_attention(const void* q, const void* k_slots, const void* v_slots, vo
     // so the map covers batch * bound rows (row_off never points past them)
     AttnMaps am;
     const long long q_rows = static_cast<long long>(batch) * rows_per_seq_bound;
-    int rc = make_attn_maps(&am, q, q_rows, k_slots, v_slots, static_cast<long long>(batch) * n_kv_heads * seq_len,
-                            n_q_heads, n_kv_heads, dtype == DKV_F16);
+    int rc = make_attn_maps(&am, q, q_rows, k_slots, v_slots, static_cast<long long>(batch) * n_kv_heads, seq_len,
+                            seq_len, n_q_heads, n_kv_heads, dtype == DKV_F16);
     if (rc) return rc;
     return attention_tc(am, o, row_off, batch, rows_per_seq_bound, seq_len, n_q_heads, n_kv_heads, 0, dtype == DKV_BF16,
                         nullptr, st);
@@ -1494,7 +1545,8 @@ int dkv_op_gemm_static(const void* x, const void* w, float* out, int rows, int n
   if (rc) return rc;
   // every float the reduction reads was written by the GEMM launch just above:
   // nothing in the shared scratch has to start at zero
-  launch_k(k_reduce_partials, std::min(4 * NUM_SMS, ceil_div(rows * n, 256)), 256, 0, st,
+  const long long elems = static_cast<long long>(rows) * n;
+  launch_k(k_reduce_partials, static_cast<int>(std::min<long long>(4 * NUM_SMS, (elems + 255) / 256)), 256, 0, st,
            static_cast<const float*>(scratch), s, stride, rows, static_cast<const int*>(nullptr), n, out);
   return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
 }

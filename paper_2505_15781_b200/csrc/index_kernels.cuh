@@ -106,13 +106,36 @@ __global__ void __launch_bounds__(256) k_compact(CompactParams p) {
   const int L = p.seq_len;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  // offsets of this sequence = number of active / head rows of the sequences before it
+  // offsets of this sequence = number of active / head rows of the sequences before it.  In the
+  // common modes these counts need no per-position predicate: all rows / generation rows / prompt
+  // rows are a product, the mask-driven set is the number of non-zero bytes of the flat mask in
+  // front of this sequence (16-byte loads), and the head rows are the masked positions of each
+  // earlier sequence's candidate range.  Greedy and the shifted variants take the general loop.
   int ca = 0, ch = 0;
-  for (int bb = 0; bb < b; ++bb) {
-    for (int pos = tid; pos < L; pos += 256) {
-      ca += is_active(p, bb, pos) ? 1 : 0;
-      ch += is_head(p, bb, pos) ? 1 : 0;
+  const bool general = p.mode == ACT_GREEDY || p.shift || p.right || p.head_from_d;
+  if (general) {
+    for (int bb = 0; bb < b; ++bb) {
+      for (int pos = tid; pos < L; pos += 256) {
+        ca += is_active(p, bb, pos) ? 1 : 0;
+        ch += is_head(p, bb, pos) ? 1 : 0;
+      }
     }
+  } else {
+    if (p.mode == ACT_FROM_MASK) {
+      const long long n = static_cast<long long>(b) * L;
+      const uint4* m16 = reinterpret_cast<const uint4*>(p.mask_src);
+      const long long n16 = (reinterpret_cast<uintptr_t>(p.mask_src) & 15) ? 0 : n / 16;   // a caller's mask may be unaligned
+      for (long long i = tid; i < n16; i += 256) {
+        const uint4 v = m16[i];
+        ca += __popc(__vcmpne4(v.x, 0u) & 0x01010101u) + __popc(__vcmpne4(v.y, 0u) & 0x01010101u) +
+              __popc(__vcmpne4(v.z, 0u) & 0x01010101u) + __popc(__vcmpne4(v.w, 0u) & 0x01010101u);
+      }
+      for (long long i = n16 * 16 + tid; i < n; i += 256) ca += p.mask_src[i] != 0 ? 1 : 0;
+    } else if (tid == 0) {
+      ca = b * (p.mode == ACT_FULL ? L : (p.mode == ACT_GEN_ONLY ? L - p.prompt_len : p.prompt_len));
+    }
+    for (int bb = 0; bb < b; ++bb)
+      for (int pos = p.cand_lo + tid; pos < p.cand_hi; pos += 256) ch += p.mask_cur[bb * L + pos] != 0 ? 1 : 0;
   }
   for (int o = 16; o > 0; o >>= 1) {
     ca += __shfl_xor_sync(0xffffffffu, ca, o);

@@ -180,22 +180,28 @@ def layer_tensor_shapes(ms: ModelShape) -> Dict[str, tuple]:
     }
 
 
+def norm_gain(seed: int, layer: int, name: str, d: int, device="cpu", spread: float = 0.1):
+    """Gain vector of one RMSNorm: 1 + spread * N(0,1) from the same counter-based generator (fp32).
+    Every norm of a model gets its own values, so a gain that is dropped, or taken from the wrong
+    norm, changes the logits."""
+    return normal_tensor(seed, layer, name, (d,), spread, "float32", device) + 1.0
+
+
 def make_weights(ms: ModelShape, seed: int = 0, dtype: str = "float32", device="cpu",
                  std: float = 0.02) -> Dict[str, object]:
     """All tensors of a model: {'embed','final_norm','head', 'layers':[{...}]}.
-    Norm gains are 1.0 (fp32).  Matrices are N(0,std) in ``dtype``."""
-    import torch
+    Matrices are N(0,std) in ``dtype``; norm gains are 1 + 0.1 * N(0,1) (fp32)."""
     w: Dict[str, object] = {}
     w["embed"] = normal_tensor(seed, -1, "embed", (ms.vocab, ms.d_model), std, dtype, device)
     w["head"] = normal_tensor(seed, -1, "head", (ms.vocab, ms.d_model), std, dtype, device)
-    w["final_norm"] = torch.ones(ms.d_model, dtype=torch.float32, device=device)
+    w["final_norm"] = norm_gain(seed, -1, "final_norm", ms.d_model, device)
     layers: List[Dict[str, object]] = []
     for l in range(ms.n_layers):
         lw = {}
         for name, shp in layer_tensor_shapes(ms).items():
             lw[name] = normal_tensor(seed, l, name, shp, std, dtype, device)
-        lw["attn_norm"] = torch.ones(ms.d_model, dtype=torch.float32, device=device)
-        lw["ffn_norm"] = torch.ones(ms.d_model, dtype=torch.float32, device=device)
+        lw["attn_norm"] = norm_gain(seed, l, "attn_norm", ms.d_model, device)
+        lw["ffn_norm"] = norm_gain(seed, l, "ffn_norm", ms.d_model, device)
         layers.append(lw)
     w["layers"] = layers
     return w

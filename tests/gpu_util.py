@@ -42,10 +42,22 @@ class ForcedRun:
     """Feeds the oracle's (x_t, M_t) of every step to the CUDA library and
     collects what it returns."""
 
-    def __init__(self, ms, model, batch, P, G, pol: O.Policy, k):
-        self.ms, self.B, self.L, self.P, self.k = ms, batch, P + G, P, k
-        self.cache = B.dkv_init_cache(model, batch, P + G, P, gpu_policy(pol, max_k=k))
+    def __init__(self, ms, model, batch, P, G, pol: O.Policy, k, fused=False, arena_fill=None):
+        """fused: also drive a second handle WITHOUT a logits buffer, i.e. through the head GEMM's
+        statistics epilogue (the path the benchmark times); its conf / pred land in conf_f / pred_f.
+        arena_fill: byte value the arenas are filled with before dkv_init_cache (None: torch.empty)."""
+        self.ms, self.B, self.L, self.P, self.k, self.score = ms, batch, P + G, P, k, pol.score
         dev = "cuda"
+
+        def arena():
+            if arena_fill is None:
+                return None
+            need = B.dkv_cache_bytes(model, batch, P + G, gpu_policy(pol, max_k=k))
+            return torch.full((need + 256,), arena_fill, dtype=torch.uint8, device=dev)
+        self.cache = B.dkv_init_cache(model, batch, P + G, P, gpu_policy(pol, max_k=k), arena=arena())
+        self.cache_f = B.dkv_init_cache(model, batch, P + G, P, gpu_policy(pol, max_k=k), arena=arena()) if fused else None
+        self.conf_f = torch.empty(batch, self.L, dtype=torch.float32, device=dev)
+        self.pred_f = torch.empty(batch, self.L, dtype=torch.int32, device=dev)
         self.conf = torch.empty(batch, self.L, dtype=torch.float32, device=dev)
         self.pred = torch.empty(batch, self.L, dtype=torch.int32, device=dev)
         self.logits = torch.zeros(batch * G, ms.vocab, dtype=torch.float32, device=dev)
@@ -64,15 +76,48 @@ class ForcedRun:
         lo, hi = traces_t[0].cand
         rows_bound = int(max(s.masked_in.sum() for s in traces_t))
         B.dkv_step(self.cache, x, m, npos, self.k, lo, hi, rows_bound, self.conf, self.pred, self.logits)
+        if self.cache_f is not None:
+            B.dkv_step(self.cache_f, x, m, npos, self.k, lo, hi, rows_bound, self.conf_f, self.pred_f, None)
         B.dkv_get_index_maps(self.cache, self.act_idx, self.row_off, self.inv)
         B.dkv_get_provenance(self.cache, self.prov)
         torch.cuda.synchronize()
         return x, m
 
 
+def score_bound(score, eps, conf_ref, p_max):
+    """How far a score may move when every logit moves by at most eps.  With |dl_i| <= eps every
+    probability moves by a factor within [e^-2eps, e^2eps] (numerator and normaliser each by e^eps):
+    the largest probability by (e^2eps - 1) p_max; the margin of the two largest (order statistics are
+    1-Lipschitz in the sup norm) by twice that; sum p log p by 2 eps + (e^2eps - 1) |sum p log p|."""
+    g = np.expm1(2.0 * eps)
+    if score == O.SCORE_MAXPROB:
+        return g * p_max
+    if score == O.SCORE_MARGIN:
+        return 2.0 * g * p_max
+    return 2.0 * eps + g * abs(conf_ref)
+
+
+def check_head_outputs(conf, pred, s, mask_id, score, eps, what):
+    """conf / pred of one sequence against the oracle's trace s, given that the logits are within
+    eps (absolute) of the oracle's: the token must agree wherever the oracle's two largest logits are
+    more than 2 eps apart, the score within score_bound (plus fp32 evaluation noise)."""
+    for j, pos in enumerate(s.head_rows):
+        l = np.array(s.logits[j], dtype=np.float64)
+        l[mask_id] = -np.inf
+        top2 = np.sort(l)[-2:]
+        if top2[1] - top2[0] > 2.0 * eps:
+            assert pred[pos] == s.pred[pos], f"{what}: token at position {pos}, step {s.t}"
+        p_max = 1.0 / np.exp(l - top2[1]).sum()
+        bound = score_bound(score, eps, s.conf[pos], p_max) + 1e-5 * abs(s.conf[pos]) + 1e-9
+        assert abs(conf[pos] - s.conf[pos]) <= bound, \
+            f"{what}: score at position {pos}, step {s.t}: {conf[pos]} vs {s.conf[pos]} (bound {bound})"
+
+
 def compare_step(run: ForcedRun, traces_t, greedy, logit_tol_abs=None, logit_tol_sigma=None):
-    """Integer outputs bit-exact; logits within the given tolerance.  Returns
-    (max abs logit error, sigma of the oracle's logits)."""
+    """Integer outputs bit-exact; logits within the given tolerance; with a sigma tolerance (16-bit
+    modes) also the scores and tokens of the head rows, within what that logit tolerance allows, on
+    the materialised-logits path and, when the run drives one, on the fused head path.  Returns
+    (max abs logit error, sigma of the oracle's logits, conf, pred)."""
     x, m = run.step(traces_t, greedy)
     L = run.L
     row_off = run.row_off.cpu().numpy()
@@ -108,4 +153,14 @@ def compare_step(run: ForcedRun, traces_t, greedy, logit_tol_abs=None, logit_tol
     if logit_tol_sigma is not None:
         assert max_err <= logit_tol_sigma * sig, \
             f"step {traces_t[0].t}: logits max-abs error {max_err} > {logit_tol_sigma} * sigma ({sig})"
+        if ref_all is not None:
+            eps = logit_tol_sigma * sig
+            conf_f, pred_f = run.conf_f.cpu().numpy(), run.pred_f.cpu().numpy()
+            for b, s in enumerate(traces_t):
+                check_head_outputs(conf[b], pred[b], s, run.ms.mask_id, run.score, eps, "materialised logits")
+                if run.cache_f is not None:
+                    check_head_outputs(conf_f[b], pred_f[b], s, run.ms.mask_id, run.score, eps, "fused head epilogue")
+                    not_head = np.ones(L, bool)
+                    not_head[s.head_rows] = False
+                    assert np.isneginf(conf_f[b][not_head]).all() and (pred_f[b][not_head] == -1).all()
     return max_err, sig, conf, pred

@@ -38,6 +38,32 @@ def test_host_only_calls():
     assert lib.dkv_model_bytes(None) == 0
 
 
+def test_a_handle_that_is_not_live_is_a_state_error():
+    """A pointer that no create call returned (or that was destroyed) is refused before anything is
+    read through it: DKV_E_STATE from every entry point that takes a handle."""
+    lib = B.load()
+    buf = ctypes.create_string_buffer(4096)
+    bogus = ctypes.c_void_p(ctypes.addressof(buf))
+    one = ctypes.c_void_p(ctypes.addressof(buf) + 64)      # stands for any non-NULL pointer argument
+    assert lib.dkv_refresh(bogus, 0) == -3
+    assert lib.dkv_status(bogus, None) == -3
+    assert lib.dkv_step(bogus, one, one, None, 1, 0, 1, -1, one, one, None, None) == -3
+    assert lib.dkv_step_host(bogus, one, one, None, 1, 0, 1, -1, None, None) == -3
+    assert lib.dkv_generate(bogus, one, one, None, 1, 0, 0, None, None) == -3
+    assert lib.dkv_get_stats(bogus, ctypes.cast(one, ctypes.POINTER(B.dkv_stats))) == -3
+    assert lib.dkv_get_provenance(bogus, one, None) == -3
+    assert lib.dkv_get_index_maps(bogus, None, None, None, None) == -3
+    assert lib.dkv_cache_slots(bogus, 0, None, None) == -3
+    assert lib.dkv_profile_enable(bogus, 1) == -3
+    assert lib.dkv_cache_destroy(bogus) == -3
+    assert lib.dkv_model_destroy(bogus) == -3
+    assert lib.dkv_cache_bytes(bogus, 1, 16, None) == 0
+    pol = B.make_policy(B.DKV_POLICY_DECODE)
+    out = ctypes.c_void_p()
+    assert lib.dkv_init_cache(bogus, 1, 16, 8, ctypes.byref(pol), one, 1 << 20, None, ctypes.byref(out)) == -3
+    assert b"state" in lib.dkv_strerror(-3)
+
+
 def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(B.dkv_model_desc) == 48
     assert ctypes.sizeof(B.dkv_policy) == 40

@@ -139,3 +139,83 @@ def test_attention_accumulator_rescale_path(rows, L, hq, hkv):
     B.dkv_op_attention(tq, tk, tv, o, row_off, 1, rows, L, hq, hkv, 128, B.DKV_F16)
     ref, valid = oracle_attention(tq, tk, tv, n_rows, row_off.cpu().numpy())
     np.testing.assert_allclose(o.float().cpu().numpy()[valid], ref[valid], atol=6 * 2.0 ** -11, rtol=6 * 2.0 ** -11)
+
+
+HD128 = synth.ModelShape(2, 256, 2, 2, 128, 512, 1000, 999)     # head_dim 128: the tcgen05 attention kernel
+
+
+@pytest.mark.parametrize("P,G", [(37, 40), (100, 92)])
+def test_step_does_not_depend_on_what_the_arena_held(P, G):
+    """Two layers, head_dim 128, a sequence length that is no multiple of the attention kernel's slot
+    tile (64 or 128), the arena filled with 0xFF bytes (NaN patterns in fp16 and fp32) before the
+    cache is initialised.  At step 1 layer 0 attends while layer 1's slots are still unwritten, and the
+    last slot tile of layer 0's last head reaches past the sequence: nothing of that may leak into
+    the result.  Compared with the oracle for a full step and two cached steps, on both head paths."""
+    ms, pol = HD128, O.Policy(O.POLICY_DECODE, 0)
+    W, model = U.build_pair(ms, 11, True)
+    prompts = synth.make_prompt(2, P, ms.vocab - 1, 11)
+    samplers = [O.Sampler(U.oracle_model(ms), W, prompts[b], G, 2, pol, None, None, "literal", keep_logits=True)
+                for b in range(2)]
+    run = U.ForcedRun(ms, model, 2, P, G, pol, 2, fused=True, arena_fill=0xFF)
+    for _ in range(3):
+        tr_t = [s.step() for s in samplers]
+        err, sig, conf, pred = U.compare_step(run, tr_t, False, logit_tol_sigma=2e-2)
+        assert np.isfinite(err)
+    assert B.dkv_status(run.cache) == 0 and B.dkv_status(run.cache_f) == 0
+
+
+def slot_tensors(cache, ms, layer, batch, L, dtype):
+    """The K and V slots of one layer as torch views [batch, kv_heads, L, head_dim] into the arena."""
+    kp, vp = B.dkv_cache_slots(cache, layer)
+    n = batch * ms.n_kv_heads * L * ms.head_dim
+    esz = torch.tensor([], dtype=dtype).element_size()
+    out = []
+    for ptr in (kp, vp):
+        off = ptr - cache.arena.data_ptr()
+        out.append(cache.arena[off:off + n * esz].view(dtype).view(batch, ms.n_kv_heads, L, ms.head_dim))
+    return out
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_cache_slot_contents_match_the_oracles_cache(bf16):
+    """Which step's K/V a position holds (Appendix A: a token's states enter the cache one step after it
+    is decoded): after a full step and two cached steps every slot of every layer is compared with the
+    oracle's position-addressed cache, stable rows (still holding an earlier step's K/V) and active rows
+    alike.  fp32 mode: 1e-5 absolute; 16-bit mode: the operand and slot rounding of fp16 (2^-11 relative
+    each, accumulated over the layers) -- 1e-2 of the tensor's rms."""
+    ms = HD128 if bf16 else dataclasses.replace(synth.tiny_shape(), n_kv_heads=2)
+    P, G, k, pol = 12, 20, 2, O.Policy(O.POLICY_DECODE, 0)
+    W, model = U.build_pair(ms, 4, bf16)
+    prompt = synth.make_prompt(1, P, ms.vocab - 1, 4)
+    sampler = O.Sampler(U.oracle_model(ms), W, prompt[0], G, k, pol, None, None, "slots", keep_logits=True)
+    run = U.ForcedRun(ms, model, 1, P, G, pol, k)
+    L = P + G
+    for _ in range(3):
+        U.compare_step(run, [sampler.step()], False, logit_tol_abs=None if bf16 else 1e-4,
+                       logit_tol_sigma=2e-2 if bf16 else None)
+    assert (sampler.cache.written_step[:P] == 1).all()          # the prompt rows still hold step 1's K/V
+    for layer in range(ms.n_layers):
+        ks, vs = slot_tensors(run.cache, ms, layer, 1, L, torch.float16 if bf16 else torch.float32)
+        for got, ref in ((ks, sampler.cache.K[layer]), (vs, sampler.cache.V[layer])):
+            g = got[0].float().cpu().numpy().transpose(1, 0, 2)          # [L, kv_heads, head_dim] like the oracle
+            tol = 1e-2 * np.sqrt(np.mean(ref * ref)) if bf16 else 1e-5
+            assert np.abs(g - ref).max() <= tol, f"layer {layer}: slot contents differ by {np.abs(g - ref).max()}"
+
+
+def test_greedy_rejects_a_change_of_k_between_steps():
+    """The window rule reads D_{t-1} with the k it was stored with."""
+    ms = synth.tiny_shape()
+    _, model = U.build_pair(ms, 0, False)
+    cache = B.dkv_init_cache(model, 1, 16, 8, B.make_policy(B.DKV_POLICY_GREEDY, window=4, max_k=2))
+    x = torch.zeros(1, 16, dtype=torch.int32, device="cuda")
+    m = torch.zeros(1, 16, dtype=torch.uint8, device="cuda")
+    m[0, 8:] = 1
+    conf = torch.empty(1, 16, device="cuda")
+    pred = torch.empty(1, 16, dtype=torch.int32, device="cuda")
+    d = torch.tensor([[8, 9]], dtype=torch.int32, device="cuda")
+    B.dkv_step(cache, x, m, d, 2, 8, 16, 8, conf, pred)
+    with pytest.raises(B.DkvError) as e:
+        B.dkv_step(cache, x, m, d, 1, 8, 16, 8, conf, pred)
+    assert e.value.status == -2
+    B.dkv_step(cache, x, m, d, 2, 8, 16, 8, conf, pred)
+    assert B.dkv_status(cache) == 0

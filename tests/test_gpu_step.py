@@ -33,7 +33,7 @@ def run_forced(ms, bf16, batch, P, G, k, pol, block=None, seed=0, with_order=Fal
     W, model = U.build_pair(ms, seed, bf16, act=act)
     order = synth.random_order(batch, P, G, k, seed) if with_order else None
     traces = oracle_traces(ms, W, batch, P, G, k, pol, block, seed, order)
-    run = U.ForcedRun(ms, model, batch, P, G, pol, k)
+    run = U.ForcedRun(ms, model, batch, P, G, pol, k, fused=bf16)     # 16-bit: both head paths, every step
     greedy = pol.kind == O.POLICY_GREEDY
     worst = 0.0
     for t in range(len(traces[0])):

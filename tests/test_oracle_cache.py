@@ -103,7 +103,6 @@ def test_active_row_totals_cubic_vs_quadratic(G, tot_vanilla, tot_decode, tot_gr
     assert c[0] == G and all(c[s] == G - s + 1 for s in range(1, G))      # #M_t + k
     assert sum(c) == G + sum(G - s + 1 for s in range(1, G)) == tot_decode
     # Greedy, window 4 around D_{t-1}; interior (no clipping) upper bound is 6 rows
-    order_mid = np.array([[(7 * s) % G] for s in range(G)]) if G % 7 else order
     cg = simulate_counts(G, 0, 1, O.Policy(O.POLICY_GREEDY, 0, window=4), order)
     assert cg[0] == G and max(cg[1:]) <= 6
     assert G + 6 * (G - 1) == tot_greedy and sum(cg) <= tot_greedy
@@ -168,8 +167,10 @@ def vanilla_logits(m, W, st):
 
 
 def test_policy_none_and_interval_one_equal_vanilla_every_step():
-    for pol in (O.Policy(O.POLICY_NONE), O.Policy(O.POLICY_DECODE, 1), O.Policy(O.POLICY_PD, 1) if False else O.Policy(O.POLICY_DECODE, 1)):
-        m, W, tr = run(pol)
+    greedy_order = (rng(9).permutation(8) + 5).reshape(8, 1)
+    for pol, order in ((O.Policy(O.POLICY_NONE), None), (O.Policy(O.POLICY_DECODE, 1), None),
+                       (O.Policy(O.POLICY_GREEDY, 1, window=2), greedy_order)):
+        m, W, tr = run(pol, order=order)
         for st in tr:
             assert len(st.active) == len(st.x_in)
             np.testing.assert_allclose(st.logits, vanilla_logits(m, W, st), atol=1e-11)
@@ -309,6 +310,22 @@ def test_cache_ratio():
     L = P + G
     expect = np.mean([0.0] + [(L - ((G - s) + 1)) / L for s in range(1, G)])
     assert abs(O.cache_ratio(tr) - expect) < 1e-15
+
+
+def test_cache_ratio_counts_prefill_rows_as_computed():
+    """PD with a prompt-only prefill pass, P = 5, G = 8 (L = 13), one token per step, a refresh every
+    4 steps.  Rows COMPUTED per step, written out by hand: step 1 computes the 5 prompt rows in the
+    prefill pass and the 8 generation rows in its own pass (13 of 13: nothing is served from the
+    cache); steps 2-4 compute the masked rows of the step before (8, 7, 6); step 5 (s = 4) is a
+    refresh of the generation rows (8); steps 6-8 compute 4, 3, 2.  The prompt rows are cache-served
+    in every step but the first.  Cache ratio = mean over steps of (13 - computed) / 13."""
+    _, _, tr = run(O.Policy(O.POLICY_PD, 4, isolated_prefill=True), G=8, P=5, keep_logits=False)
+    computed = [13, 8, 7, 6, 8, 4, 3, 2]
+    assert [len(s.active) + s.prefilled for s in tr] == computed
+    assert abs(O.cache_ratio(tr) - (0 + 5 + 6 + 7 + 5 + 9 + 10 + 11) / (8 * 13)) < 1e-15
+    # the same policy without the separate pass computes the same 13 rows at step 1 in one pass
+    _, _, tr2 = run(O.Policy(O.POLICY_PD, 4), G=8, P=5, keep_logits=False)
+    assert [len(s.active) for s in tr2] == computed and O.cache_ratio(tr2) == O.cache_ratio(tr)
 
 
 def test_greedy_uses_given_order_and_bounded_rows():
