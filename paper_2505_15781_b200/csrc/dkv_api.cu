@@ -29,7 +29,8 @@ using namespace dkv;
 
 namespace {
 
-constexpr int NUM_SMS = 148;
+constexpr int NUM_SMS = 148;            // B200; the cost models are calibrated for it
+constexpr int MAX_TILE_COUNTERS = 256;  // arrival counters of the fused GEMM tails (one per weight tile x row tile)
 constexpr int N_BOX = 16;   // row boxes of 16, 32, ..., 256 rows
 inline int box_rows(int i) { return 16 * (i + 1); }
 
@@ -61,6 +62,19 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
   cfg.attrs = attr;
   cfg.numAttrs = use_pdl ? 1 : 0;
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// SMs of the current device (looked up once per device): what bounds a launch whose CTAs wait for each other.
+inline int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  if (!cached[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 1;
+    cached[dev] = n;
+  }
+  return cached[dev];
 }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -210,8 +224,8 @@ struct dkv_model {
   int d_q, d_kv, n_qkv;
   size_t esize;   // bytes per weight element
   size_t asize;   // bytes per activation / cache element
-  int gu_blk;     // > 0: the gate/up copy is regrouped [blk gate | blk up] per tile (SwiGLU in the GEMM epilogue);
-                  // 128 = one CTA's tile, 256 = a CTA pair's tile (the pair kernel runs the fused launch)
+  int gu_blk;     // 128: the gate/up copy is regrouped [128 gate | 128 up] per 256 rows (SwiGLU in the GEMM epilogue); 0: not
+  bool gu_pair;   // the standalone SwiGLU launch runs on CTA pairs (d_ffn a multiple of 256)
 };
 
 namespace {
@@ -246,6 +260,9 @@ struct Arena {
   float* st_m2;
   float* st_t;
   float* part;
+  float* ssq;                    // [ceil(d_model / 128)][r_cap]: partial sums of squares of the residual rows
+  float* head_rs;                // [h_cap]: 1 / RMS of each head row
+  unsigned int* tile_cnt;        // [MAX_TILE_COUNTERS]: arrival counters of the fused GEMM tails
   float* conf_i;
   int32_t* pred_i;
   int32_t* tok_stage;
@@ -320,6 +337,9 @@ void carve(const dkv_model* m, const Dims& d, uint8_t* base, Arena* a) {
     a->st_t = reinterpret_cast<float*>(take(groups * d.h_cap * 4));
   }
   a->part = reinterpret_cast<float*>(take(d.part_rows * d.n_max * 4));
+  a->ssq = reinterpret_cast<float*>(take(static_cast<size_t>((md.d_model + 127) / 128) * d.r_cap * 4));
+  a->head_rs = reinterpret_cast<float*>(take(d.h_cap * 4));
+  a->tile_cnt = reinterpret_cast<unsigned int*>(take(MAX_TILE_COUNTERS * 4));
   a->conf_i = reinterpret_cast<float*>(take(BL * 4));
   a->pred_i = reinterpret_cast<int32_t*>(take(BL * 4));
   a->tok_stage = reinterpret_cast<int32_t*>(take(BL * 4));
@@ -347,6 +367,8 @@ struct dkv_cache {
   AttnMaps attn_maps;            // tcgen05 attention (head_dim 128, 16-bit modes): all seq_len slots attended
   AttnMaps attn_maps_prompt;     // the same buffers with the slot extent cut at the prompt (isolated prefill pass)
   bool attn_tc;
+  int fuse_tails;        // bit 0: RoPE / K/V scatter inside the QKV GEMM; bit 1: residual / norm statistics inside
+                         // the O and down GEMMs (one-wave launches)
   int step;              // steps run so far
   int last_refresh;      // step number of the last full / generation-only step
   int pending_refresh;   // -1 none, else DKV_REFRESH_*
@@ -491,14 +513,12 @@ int env_int(const char* name, int dflt) {
 // fraction of CTA slots the units fill in their last wave, plus the fp32
 // partials written and read back (they mostly stay in L2, hence the weight 1/2).
 // Sweeps over the four LLaDA-shaped projections showed total time (GEMM plus
-// the row kernel that reduces the partials) flat within 10 % around this choice.
+// the reduction of the partials) flat within 10 % around this choice.
 int choose_splits(int n, int k, int r_bound, const GemmTcPlan& plan, long long part_rows) {
-  static const int forced = env_int("DKV_GEMM_SPLITS", 0);
   const int tiles = ceil_div(n, GEMM_BM * plan.halves) * ceil_div(r_bound, plan.br);
   const int kb_total = ceil_div(k, GEMM_BK);
   int s_max = std::min(16, std::max(1, kb_total / 4));
   s_max = static_cast<int>(std::min<long long>(s_max, std::max<long long>(1, part_rows / std::max(1, r_bound))));
-  if (forced > 0) return std::max(1, std::min(forced, s_max));
   const double slots = static_cast<double>(plan.ctas_per_sm) * NUM_SMS;
   const double w_bytes = 2.0 * n * static_cast<double>(k);
   int best = 1;
@@ -525,41 +545,89 @@ struct HeadStats {   // vocabulary-head mode of the GEMM epilogue
   float* st_t;
 };
 
-// out (fp32 partials) [splits][r_bound * n]; returns splits and stride through the pointers
+// Per-row scale of a GEMM's result: the RMSNorm of its operand, applied after the product.
+struct RowScale {
+  const float* src = nullptr;   // NULL: no scale
+  int parts = 0;                // > 0: src = [parts][ld] partial sums of squares; 0: src = ready factors
+  long long ld = 0;
+  int d = 1;
+  float eps = 0.f;
+};
+
+// Row epilogue fused into the GEMM across the CTAs of a weight tile (FUSE_RESID / FUSE_QKV).
+struct FusedTail {
+  int mode = FUSE_NONE;
+  unsigned int* tile_cnt = nullptr;
+  float* h = nullptr;
+  const float* gain = nullptr;
+  void* xn_out = nullptr;
+  float* ssq_out = nullptr;
+  long long ssq_ld = 0;
+  const int32_t* act_idx = nullptr;
+  const float2* rope_tab = nullptr;
+  int seq_len = 0, n_q_heads = 0, n_kv_heads = 0, head_dim = 0;
+  void* q_out = nullptr;
+  void* k_slots = nullptr;
+  void* v_slots = nullptr;
+};
+
+struct GemmOpts {
+  int forced_splits = 0;
+  bool w_static = true;
+  const HeadStats* head = nullptr;
+  void* swiglu_out = nullptr;
+  int ld_u = 0;
+  const CUtensorMap* xmaps_half = nullptr;   // [N_BOX] boxes of half the rows: run on CTA pairs
+  int row_tiles = 0;                         // > 0: this many row tiles instead of ceil(rows / 256)
+  RowScale scale;
+  FusedTail tail;                            // applied only when the launch is one wave (see *fused_out)
+};
+
+// out (fp32 partials) [splits][r_bound * n]; returns splits and stride through the pointers.  When a
+// fused tail is asked for and every unit gets a CTA of its own (units <= SMs, so that the CTAs of a
+// tile can wait for each other), the kernel runs it and *fused_out is true; otherwise the partials
+// are left in `out` for a row kernel.
 int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, int k, int r_bound,
-            const int* r_dev, float* out, long long part_rows, int forced_splits, int* status, bool x_bf16,
-            cudaStream_t st, int* splits_out, long long* stride_out, bool w_static = true,
-            const HeadStats* head = nullptr, void* swiglu_out = nullptr, int ld_u = 0,
-            const CUtensorMap* xmaps_half = nullptr /*[N_BOX] boxes of half the rows: run on CTA pairs*/,
-            int row_tiles = 0 /*> 0: this many row tiles instead of ceil(rows / 256)*/) {
+            const int* r_dev, float* out, long long part_rows, int* status, bool x_bf16, cudaStream_t st,
+            int* splits_out, long long* stride_out, const GemmOpts& o = GemmOpts(), bool* fused_out = nullptr) {
   static PerDeviceOnce attr_once;
   if (attr_once.need()) {
     if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return DKV_E_CUDA;
   }
-  if (xmaps_half) {
+  if (fused_out) *fused_out = false;
+  GemmTcParams p;
+  memset(&p, 0, sizeof(p));
+  p.n = n;
+  p.r_bound = r_bound;
+  p.r_dev = r_dev;
+  p.out = out;
+  p.split_stride = static_cast<long long>(r_bound) * n;
+  p.ldo = n;
+  p.status = status;
+  p.x_bf16 = x_bf16 ? 1 : 0;
+  p.w_static = o.w_static ? 1 : 0;
+  p.swiglu_out = o.swiglu_out;
+  p.ld_u = o.ld_u;
+  p.mask_id = -1;
+  p.rs_src = o.scale.src;
+  p.rs_parts = o.scale.parts;
+  p.rs_ld = o.scale.ld;
+  p.rs_inv_d = 1.f / static_cast<float>(o.scale.d);
+  p.rs_eps = o.scale.eps;
+  const int kb_total = ceil_div(k, GEMM_BK);
+  p.kb_total = kb_total;
+  if (o.xmaps_half) {
     // CTA pairs (cta_group::2): 512-row weight tiles, each CTA stages half of the row tile.  Used for
     // the unsplit SwiGLU launch, whose few CTAs are bound by the operand bytes an SM can take in.
-    const int bi = row_tiles > 0 ? std::min(std::max(ceil_div(ceil_div(r_bound, row_tiles), 16) - 1, 0), N_BOX - 1)
-                                 : pick_box(r_bound);
+    const int bi = o.row_tiles > 0 ? std::min(std::max(ceil_div(ceil_div(r_bound, o.row_tiles), 16) - 1, 0), N_BOX - 1)
+                                   : pick_box(r_bound);
     const int br = box_rows(bi);
     GemmTcPlan plan = gemm_tc2_plan(br);
-    const int kb_total = ceil_div(k, GEMM_BK);
-    const int splits = std::max(1, std::min(forced_splits, kb_total));
-    GemmTcParams p;
-    memset(&p, 0, sizeof(p));
-    p.n = n;
-    p.kb_total = kb_total;
+    const int splits = std::max(1, std::min(o.forced_splits, kb_total));
     p.kb_per_split = ceil_div(kb_total, splits);
     p.splits = splits;
-    p.r_bound = r_bound;
-    p.r_dev = r_dev;
-    p.out = out;
-    p.split_stride = static_cast<long long>(r_bound) * n;
-    p.ldo = n;
-    p.status = status;
-    p.x_bf16 = x_bf16 ? 1 : 0;
     p.br = br;
     p.halves = 2;
     p.stages = plan.stages;
@@ -569,50 +637,30 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
     p.tmem_cols = plan.tmem_cols;
     p.r_tiles = ceil_div(r_bound, br);
     p.units = ceil_div(n, GEMM2_TILE_ROWS) * p.r_tiles * splits;
-    p.w_static = w_static ? 1 : 0;
-    p.swiglu_out = swiglu_out;
-    p.ld_u = ld_u;
-    p.mask_id = -1;
     const int grid = 2 * std::min(p.units, NUM_SMS / 2);
-    launch_k(k_gemm_tc2, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps_half[bi], p);
+    launch_k(k_gemm_tc2, grid, GEMM_THREADS, plan.smem_bytes, st, tw, o.xmaps_half[bi], p);
     *splits_out = splits;
     *stride_out = p.split_stride;
     return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
   }
-  static const int env_halves = env_int("DKV_GEMM_HALVES", 0);
-  static const int env_ctas = env_int("DKV_GEMM_CTAS", 0);
-  int halves = env_halves > 0 ? env_halves : 2;
+  int halves = 2;
   if (n <= GEMM_BM) halves = 1;
-  if (swiglu_out) halves = 2;
-  int ctas = env_ctas > 0 ? env_ctas : 1;
   int bi = pick_box(r_bound);
   int multi_splits = 0;
-  static const int env_mt = env_int("DKV_GEMM_MULTITILE", 1);
-  if (env_mt && r_bound > 256 && halves == 2 && forced_splits <= 0 && !head && !swiglu_out) {
+  if (r_bound > 256 && halves == 2 && o.forced_splits <= 0 && !o.head && !o.swiglu_out) {
     int t = 0;
     choose_multi_tile(n, k, r_bound, part_rows, &t, &multi_splits);
     bi = std::min(std::max(ceil_div(ceil_div(r_bound, t), 16) - 1, 0), N_BOX - 1);
   }
   const int br = box_rows(bi);
-  GemmTcPlan plan = gemm_tc_plan(br, halves, ctas);
-  if (plan.ctas_per_sm == 1 && plan.smem_bytes < 116 * 1024) plan.smem_bytes = 116 * 1024;  // keep the SM to one CTA
-  int splits = forced_splits > 0 ? forced_splits
-                                 : (multi_splits > 0 ? multi_splits : choose_splits(n, k, r_bound, plan, part_rows));
-  const int kb_total = ceil_div(k, GEMM_BK);
+  GemmTcPlan plan = gemm_tc_plan(br, halves, 1);
+  if (plan.smem_bytes < 116 * 1024) plan.smem_bytes = 116 * 1024;  // keep the SM to one CTA
+  int splits = o.forced_splits > 0 ? o.forced_splits
+                                   : (multi_splits > 0 ? multi_splits : choose_splits(n, k, r_bound, plan, part_rows));
   splits = std::min(splits, kb_total);
   while (splits > 1 && (splits - 1) * ceil_div(kb_total, splits) >= kb_total) --splits;
-  GemmTcParams p;
-  p.n = n;
-  p.kb_total = kb_total;
   p.kb_per_split = ceil_div(kb_total, splits);
   p.splits = splits;
-  p.r_bound = r_bound;
-  p.r_dev = r_dev;
-  p.out = out;
-  p.split_stride = static_cast<long long>(r_bound) * n;
-  p.ldo = n;
-  p.status = status;
-  p.x_bf16 = x_bf16 ? 1 : 0;
   p.br = br;
   p.halves = plan.halves;
   p.stages = plan.stages;
@@ -622,17 +670,36 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
   p.tmem_cols = plan.tmem_cols;
   p.r_tiles = ceil_div(r_bound, br);
   p.units = ceil_div(n, GEMM_BM * plan.halves) * p.r_tiles * splits;
-  p.w_static = w_static ? 1 : 0;
-  p.swiglu_out = swiglu_out;
-  p.ld_u = ld_u;
-  p.head_mode = head ? 1 : 0;
-  p.mask_id = head ? head->mask_id : -1;
-  p.st_max = head ? head->st_max : nullptr;
-  p.st_sum = head ? head->st_sum : nullptr;
-  p.st_arg = head ? head->st_arg : nullptr;
-  p.st_m2 = head ? head->st_m2 : nullptr;
-  p.st_t = head ? head->st_t : nullptr;
-  const int grid = std::min(p.units, plan.ctas_per_sm * NUM_SMS);
+  p.head_mode = o.head ? 1 : 0;
+  p.mask_id = o.head ? o.head->mask_id : -1;
+  p.st_max = o.head ? o.head->st_max : nullptr;
+  p.st_sum = o.head ? o.head->st_sum : nullptr;
+  p.st_arg = o.head ? o.head->st_arg : nullptr;
+  p.st_m2 = o.head ? o.head->st_m2 : nullptr;
+  p.st_t = o.head ? o.head->st_t : nullptr;
+  const int sms = sm_count();
+  const int grid = std::min(p.units, sms);
+  // the CTAs of a tile wait for each other in the fused tail: every unit needs a resident CTA of its own
+  if (o.tail.mode != FUSE_NONE && p.units <= sms && p.units <= MAX_TILE_COUNTERS) {
+    const FusedTail& t = o.tail;
+    p.fuse_mode = t.mode;
+    p.tile_cnt = t.tile_cnt;
+    p.h = t.h;
+    p.gain = t.gain;
+    p.xn_out = t.xn_out;
+    p.ssq_out = t.ssq_out;
+    p.ssq_ld = t.ssq_ld;
+    p.act_idx = t.act_idx;
+    p.rope_tab = t.rope_tab;
+    p.seq_len = t.seq_len;
+    p.n_q_heads = t.n_q_heads;
+    p.n_kv_heads = t.n_kv_heads;
+    p.head_dim = t.head_dim;
+    p.q_out = t.q_out;
+    p.k_slots = t.k_slots;
+    p.v_slots = t.v_slots;
+    if (fused_out) *fused_out = true;
+  }
   launch_k(k_gemm_tc, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps[bi], p);
   *splits_out = splits;
   *stride_out = p.split_stride;
@@ -682,8 +749,6 @@ int attention_mma_dh(const T* q, const T* ks, const T* vs, T* o, const int32_t* 
 template <typename T>
 int attention_16(const T* q, const T* ks, const T* vs, T* o, const int32_t* row_off, int batch, int rows_bound,
                  int seq_len, int hq, int hkv, int dh, cudaStream_t st, int kv_stride = 0) {
-  static const int use_simt = env_int("DKV_ATTN_SIMT", 0);
-  if (use_simt) return attention_simt<T>(q, ks, vs, o, row_off, batch, rows_bound, seq_len, hq, hkv, dh, st, kv_stride);
   if (dh == 128) return attention_mma_dh<128, T>(q, ks, vs, o, row_off, batch, rows_bound, seq_len, hq, hkv, st, kv_stride);
   if (dh == 64) return attention_mma_dh<64, T>(q, ks, vs, o, row_off, batch, rows_bound, seq_len, hq, hkv, st, kv_stride);
   return DKV_E_UNSUPPORTED;
@@ -731,22 +796,84 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
   const int kv_count = plan.kv_count > 0 ? plan.kv_count : dm.L;
   int rc;
 
+  // 16-bit modes: the operand of a projection that follows an RMSNorm is h .* gain, and the GEMM divides
+  // by the row's RMS in its epilogue (`sc`: where the sums of squares of the current operand rows are).
+  // The check mode keeps the normalised operand (its plain FMA GEMM has no epilogue).
+  RowScale sc;
+  float* const ssq = bf16 ? a.ssq : nullptr;
+  const long long ssq_ld = dm.r_cap;
+  auto scale_from = [&](int parts) {
+    sc.src = a.ssq;
+    sc.parts = parts;
+    sc.ld = ssq_ld;
+    sc.d = d;
+    sc.eps = md.rms_eps;
+  };
+
   auto gemm = [&](int cls, const void* w, const CUtensorMap* tw, XBuf xb, const void* x, int n, int k, int rb,
-                  const int* rdev, float* out, int* splits, long long* stride) -> int {
+                  const int* rdev, float* out, int* splits, long long* stride, const GemmOpts& o = GemmOpts(),
+                  bool* fused = nullptr) -> int {
     const double bytes = (static_cast<double>(n) * k + static_cast<double>(rb) * k) * es + 4.0 * rb * n;
     Launch l(c, st, cls, bytes, 2.0 * rb * n * static_cast<double>(k));
-    if (bf16) return gemm_tc(*tw, c->xmaps[xb], n, k, rb, rdev, out, dm.part_rows, 0, a.status, x_bf16, st, splits, stride);
+    if (fused) *fused = false;
+    if (bf16) return gemm_tc(*tw, c->xmaps[xb], n, k, rb, rdev, out, dm.part_rows, a.status, x_bf16, st, splits, stride, o, fused);
     *splits = 1;
     *stride = 0;
     return gemm_f32(static_cast<const float*>(x), static_cast<const float*>(w), n, k, rb, rdev, out, st);
+  };
+  // residual + norm around the O and down projections: fused into the GEMM when the launch is one wave
+  auto resid_opts = [&](const float* gain) {
+    GemmOpts o;
+    if (c->fuse_tails & 2) {
+      o.tail.mode = FUSE_RESID;
+      o.tail.tile_cnt = a.tile_cnt;
+      o.tail.h = a.h;
+      o.tail.gain = gain;
+      o.tail.xn_out = a.xn;
+      o.tail.ssq_out = a.ssq;
+      o.tail.ssq_ld = ssq_ld;
+    }
+    return o;
+  };
+  auto resid_after = [&](bool fused, int splits, long long stride, const float* gain) {
+    if (fused) {
+      scale_from(ceil_div(d, d <= GEMM_BM ? GEMM_BM : 2 * GEMM_BM));   // one partial sum per weight tile
+      return;
+    }
+    Launch lk(c, st, PC_RESID_NORM, R * d * (4.0 * splits + 8.0 + es), 0);
+    launch_k((k_resid_norm<T>), R, 256, 0, st, a.h, a.part, splits, stride, r_dev, gain, md.rms_eps, d,
+             static_cast<T*>(a.xn), ssq);
+    scale_from(1);
   };
 
   {
     Launch l(c, st, PC_EMBED, R * d * (es + 4.0 + es), 0);
     launch_k((k_embed_norm<TW, T>), R, 256, 0, st, static_cast<const TW*>(m->embed), tokens, a.act_idx, r_dev,
-                                        m->layers[0].attn_norm, md.rms_eps, d, a.h, static_cast<T*>(a.xn));
+                                        m->layers[0].attn_norm, md.rms_eps, d, a.h, static_cast<T*>(a.xn), ssq);
+    scale_from(1);
   }
+  if (!bf16) sc = RowScale();
   const size_t slot_layer = static_cast<size_t>(dm.B) * md.n_kv_heads * dm.L * md.head_dim;
+  auto qkv_opts = [&](int l) {
+    GemmOpts o;
+    o.scale = sc;
+    // (with several row tiles the launch is unsplit and compute-bound; there a tail through scratch
+    // costs more than the row kernel that overlaps with the next launch's weight prefetch)
+    if ((c->fuse_tails & 1) && R <= 256) {
+      o.tail.mode = FUSE_QKV;
+      o.tail.tile_cnt = a.tile_cnt;
+      o.tail.act_idx = a.act_idx;
+      o.tail.rope_tab = a.rope_tab;
+      o.tail.seq_len = dm.L;
+      o.tail.n_q_heads = md.n_q_heads;
+      o.tail.n_kv_heads = md.n_kv_heads;
+      o.tail.head_dim = md.head_dim;
+      o.tail.q_out = a.qb;
+      o.tail.k_slots = static_cast<T*>(a.k_slots) + l * slot_layer;
+      o.tail.v_slots = static_cast<T*>(a.v_slots) + l * slot_layer;
+    }
+    return o;
+  };
   for (int l = 0; l < md.n_layers; ++l) {
     const dkv_layer_weights& lw = m->layers[l];
     const LayerMaps* lm = bf16 ? &m->maps[l] : nullptr;
@@ -754,9 +881,11 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     T* vs = static_cast<T*>(a.v_slots) + l * slot_layer;
     int splits;
     long long stride;
-    rc = gemm(PC_GEMM_QKV, lw.wqkv, lm ? &lm->wqkv : nullptr, XB_XN, a.xn, nqkv, d, R, r_dev, a.part, &splits, &stride);
+    bool fused;
+    rc = gemm(PC_GEMM_QKV, lw.wqkv, lm ? &lm->wqkv : nullptr, XB_XN, a.xn, nqkv, d, R, r_dev, a.part, &splits, &stride,
+              qkv_opts(l), &fused);
     if (rc) return rc;
-    {
+    if (!fused) {
       Launch lk(c, st, PC_QKV_POST, R * (nqkv * 4.0 * splits + nqkv * es), 0);
       const int units = (md.n_q_heads + md.n_kv_heads) * (md.head_dim / 8) + dkv / 4;
       // few enough blocks that the whole grid is resident at once: a kernel launched behind it with
@@ -779,21 +908,19 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
                            md.head_dim, st, dm.L);
       if (rc) return rc;
     }
-    rc = gemm(PC_GEMM_O, lw.wo, lm ? &lm->wo : nullptr, XB_AO, a.ao, d, dq, R, r_dev, a.part, &splits, &stride);
+    const float* next_gain = (l + 1 < md.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
+    rc = gemm(PC_GEMM_O, lw.wo, lm ? &lm->wo : nullptr, XB_AO, a.ao, d, dq, R, r_dev, a.part, &splits, &stride,
+              resid_opts(lw.ffn_norm), &fused);
     if (rc) return rc;
-    {
-      Launch lk(c, st, PC_RESID_NORM, R * d * (4.0 * splits + 8.0 + es), 0);
-      launch_k((k_resid_norm<T>), R, 256, 0, st, a.h, a.part, splits, stride, r_dev, lw.ffn_norm, md.rms_eps, d,
-                                          static_cast<T*>(a.xn));
-    }
+    resid_after(fused, splits, stride, lw.ffn_norm);
     // The SwiGLU epilogue needs the whole K range in one unit (no split-K).  With one row tile that
     // wins although the 2f/256 units may fill the SMs badly (no partials, one launch less); with more
     // row tiles only when the units come out as nearly whole waves.
-    const int gu_workers = m->gu_blk == 256 ? NUM_SMS / 2 : NUM_SMS;           // CTA pairs or CTAs
-    const int gu_tiles_n = ceil_div(2 * f, 2 * std::max(m->gu_blk, 128));
+    const int gu_workers = m->gu_pair ? NUM_SMS / 2 : NUM_SMS;                  // CTA pairs or CTAs
+    const int gu_tiles_n = ceil_div(2 * f, m->gu_pair ? GEMM2_TILE_ROWS : 2 * GEMM_BM);
     int gu_rt = ceil_div(R, 256);                                              // row tiles of the fused launch
     double gu_fill = 0.0;
-    for (int t = ceil_div(R, 256); t <= ceil_div(R, 256) + (m->gu_blk == 256 && R > 256 ? 1 : 0); ++t) {
+    for (int t = ceil_div(R, 256); t <= ceil_div(R, 256) + (m->gu_pair && R > 256 ? 1 : 0); ++t) {
       const int units = gu_tiles_n * t;                                        // one more, narrower tile may
       const double fill = units / (std::ceil(units / static_cast<double>(gu_workers)) * gu_workers);   // fill the waves
       if (fill > gu_fill + 0.1) {
@@ -806,39 +933,48 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       // the epilogue, the product written once as 16-bit
       const double bytes = (2.0 * f * d + static_cast<double>(R) * d) * es + static_cast<double>(R) * f * es;
       Launch lk(c, st, PC_GEMM_GU, bytes, 4.0 * R * f * static_cast<double>(d));
-      rc = gemm_tc(lm->wgu, c->xmaps[XB_XN], 2 * f, d, R, r_dev, a.part, dm.part_rows, 1, a.status, x_bf16, st, &splits,
-                   &stride, true, nullptr, a.ub, f, m->gu_blk == 256 ? c->xmaps_half : nullptr,
-                   R > 256 ? gu_rt : 0);
+      GemmOpts o;
+      o.forced_splits = 1;
+      o.scale = sc;
+      o.swiglu_out = a.ub;
+      o.ld_u = f;
+      o.xmaps_half = m->gu_pair ? c->xmaps_half : nullptr;
+      o.row_tiles = R > 256 ? gu_rt : 0;
+      rc = gemm_tc(lm->wgu, c->xmaps[XB_XN], 2 * f, d, R, r_dev, a.part, dm.part_rows, a.status, x_bf16, st, &splits,
+                   &stride, o);
       if (rc) return rc;
     } else {
-      rc = gemm(PC_GEMM_GU, lw.wgu, lm ? &lm->wgu : nullptr, XB_XN, a.xn, 2 * f, d, R, r_dev, a.part, &splits, &stride);
+      GemmOpts o;
+      o.scale = sc;
+      rc = gemm(PC_GEMM_GU, lw.wgu, lm ? &lm->wgu : nullptr, XB_XN, a.xn, 2 * f, d, R, r_dev, a.part, &splits, &stride, o);
       if (rc) return rc;
       Launch lk(c, st, PC_SWIGLU, R * f * (8.0 * splits + es), 0);
       dim3 grid(R, std::max(1, std::min(ceil_div(f / 4, 256), 1024 / std::max(R, 1))));
       launch_k((k_swiglu<T>), grid, 256, 0, st, a.part, splits, stride, r_dev, f, bf16 ? m->gu_blk : 0,
                static_cast<T*>(a.ub));
     }
-    rc = gemm(PC_GEMM_DOWN, lw.wd, lm ? &lm->wd : nullptr, XB_U, a.ub, d, f, R, r_dev, a.part, &splits, &stride);
+    rc = gemm(PC_GEMM_DOWN, lw.wd, lm ? &lm->wd : nullptr, XB_U, a.ub, d, f, R, r_dev, a.part, &splits, &stride,
+              resid_opts(next_gain), &fused);
     if (rc) return rc;
-    {
-      const float* gain = (l + 1 < md.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
-      Launch lk(c, st, PC_RESID_NORM, R * d * (4.0 * splits + 8.0 + es), 0);
-      launch_k((k_resid_norm<T>), R, 256, 0, st, a.h, a.part, splits, stride, r_dev, gain, md.rms_eps, d,
-                                          static_cast<T*>(a.xn));
-    }
+    resid_after(fused, splits, stride, next_gain);
   }
   if (H <= 0) return DKV_OK;
   {
     Launch lk(c, st, PC_HEAD_STATS, 2.0 * H * d * es, 0);
-    launch_k((k_head_gather<T>), H, 256, 0, st, static_cast<const T*>(a.xn), a.head_row, h_dev, d, static_cast<T*>(a.xh));
+    launch_k((k_head_gather<T>), H, 256, 0, st, static_cast<const T*>(a.xn), a.head_row, h_dev, d, static_cast<T*>(a.xh),
+             static_cast<const float*>(bf16 ? sc.src : nullptr), sc.parts, sc.ld, md.rms_eps, a.head_rs);
+  }
+  RowScale head_sc;
+  if (bf16) {
+    head_sc.src = a.head_rs;     // ready factors, one per head row
+    head_sc.d = d;
   }
   // 16-bit modes, no logits requested: the head GEMM's epilogue reduces every 32 token ids to
   // (max, argmax, sum exp) with warp shuffles and a small kernel combines them; the logits are
   // never written.  Otherwise (check mode, or the caller wants the logits) they are materialised.
-  static const int env_fuse_head = env_int("DKV_FUSE_HEAD", 1);
   // (the warp-shuffle reduction costs time in proportion to the head rows: with many of them the
   // GEMM is compute-bound and writing the logits is the cheaper way)
-  if (bf16 && !logits_dbg && env_fuse_head && H <= 128) {
+  if (bf16 && !logits_dbg && H <= 128) {
     int splits;
     long long stride;
     const int score = c->policy.score;
@@ -846,8 +982,12 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     {
       const double bytes = (static_cast<double>(md.vocab) * d + static_cast<double>(H) * d) * es;
       Launch lk(c, st, PC_GEMM_HEAD, bytes, 2.0 * H * md.vocab * static_cast<double>(d));
-      rc = gemm_tc(m->head_map, c->xmaps[XB_XH], md.vocab, d, H, h_dev, nullptr, dm.part_rows, 1, a.status, x_bf16, st,
-                   &splits, &stride, true, &hs);
+      GemmOpts o;
+      o.forced_splits = 1;
+      o.head = &hs;
+      o.scale = head_sc;
+      rc = gemm_tc(m->head_map, c->xmaps[XB_XH], md.vocab, d, H, h_dev, nullptr, dm.part_rows, a.status, x_bf16, st,
+                   &splits, &stride, o);
       if (rc) return rc;
     }
     Launch lk(c, st, PC_HEAD_STATS, 24.0 * H * ((md.vocab + 31) / 32), 0);
@@ -863,8 +1003,11 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     const double bytes = (static_cast<double>(md.vocab) * d + static_cast<double>(H) * d) * es + 4.0 * H * md.vocab;
     Launch lk(c, st, PC_GEMM_HEAD, bytes, 2.0 * H * md.vocab * static_cast<double>(d));
     if (bf16) {
-      rc = gemm_tc(m->head_map, c->xmaps[XB_XH], md.vocab, d, H, h_dev, logits, dm.part_rows, 1, a.status, x_bf16, st,
-                   &splits, &stride);
+      GemmOpts o;
+      o.forced_splits = 1;
+      o.scale = head_sc;
+      rc = gemm_tc(m->head_map, c->xmaps[XB_XH], md.vocab, d, H, h_dev, logits, dm.part_rows, a.status, x_bf16, st,
+                   &splits, &stride, o);
     } else {
       rc = gemm_f32(static_cast<const float*>(a.xh), static_cast<const float*>(m->head), md.vocab, d, H, h_dev,
                     logits, st);
@@ -1086,10 +1229,8 @@ int dkv_model_create(const dkv_model_desc* desc, const dkv_weights* w, void* are
       k_bf16_to_f16<<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), dst, n_elem);
       return dst;
     };
-    static const int env_gu = env_int("DKV_FUSE_SWIGLU", 1);
-    static const int env_pair = env_int("DKV_GEMM_2CTA", 1);
-    m->gu_blk = 0;
-    if (f16 && env_gu && desc->d_ffn % 128 == 0) m->gu_blk = (env_pair && desc->d_ffn % 256 == 0) ? 256 : 128;
+    m->gu_blk = (f16 && desc->d_ffn % 128 == 0) ? 128 : 0;
+    m->gu_pair = m->gu_blk && desc->d_ffn % 256 == 0;
     m->maps.resize(desc->n_layers);
     int rc = DKV_OK;
     const long long d = desc->d_model, f = desc->d_ffn;
@@ -1176,9 +1317,8 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
       if (!rc) rc = make_tmap(&c->xmaps[XB_U][i], a.ub, c->dims.r_cap, md.d_ffn, box_rows(i), h);
       if (!rc) rc = make_tmap(&c->xmaps[XB_XH][i], a.xh, c->dims.h_cap, md.d_model, box_rows(i), h);
     }
-    static const int env_attn_tc = env_int("DKV_ATTN_TC", 1);
     c->attn_tc = false;
-    if (!rc && md.head_dim == ATC_DH && env_attn_tc && md.n_q_heads / md.n_kv_heads <= ATC_M) {
+    if (!rc && md.head_dim == ATC_DH && md.n_q_heads / md.n_kv_heads <= ATC_M) {
       const long long kv_heads = static_cast<long long>(md.n_layers) * batch * md.n_kv_heads;
       const bool h16 = md.act_dtype == DKV_F16;
       rc = make_attn_maps(&c->attn_maps, a.qb, c->dims.r_cap, a.k_slots, a.v_slots, kv_heads, seq_len, seq_len,
@@ -1195,6 +1335,7 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   }
   const size_t BL = static_cast<size_t>(batch) * seq_len;
   cudaMemsetAsync(a.status, 0, 256, st);
+  cudaMemsetAsync(a.tile_cnt, 0, MAX_TILE_COUNTERS * 4, st);
   cudaMemsetAsync(a.written_step, 0, BL * 4, st);
   cudaMemsetAsync(a.mask_buf[0], 0, BL, st);
   cudaMemsetAsync(a.mask_buf[1], 0, BL, st);
@@ -1214,6 +1355,8 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
     delete c;
     return DKV_E_CUDA;
   }
+  // read per handle (not once per process), so that a test can build handles of both kinds
+  c->fuse_tails = env_int("DKV_FUSE_TAILS", 3);
   c->step = 0;
   c->last_refresh = 1;
   c->pending_refresh = -1;
@@ -1436,8 +1579,11 @@ int dkv_op_gemm(const void* x, const void* w, float* out, int rows, int n, int k
   int s;
   long long stride;
   const long long part_rows = std::max(rows, 2048);
-  rc = gemm_tc(tw, tx, n, k, rows, nullptr, static_cast<float*>(workspace), part_rows, splits, nullptr, dtype == DKV_BF16,
-               st, &s, &stride, /*w_static=*/false);
+  GemmOpts o;
+  o.forced_splits = splits;
+  o.w_static = false;
+  rc = gemm_tc(tw, tx, n, k, rows, nullptr, static_cast<float*>(workspace), part_rows, nullptr, dtype == DKV_BF16, st, &s,
+               &stride, o);
   if (rc || !out) return rc;   // out == NULL: the split-K partials stay in the workspace
   const long long elems = static_cast<long long>(rows) * n;
   launch_k(k_reduce_partials, static_cast<int>(std::min<long long>(4 * NUM_SMS, (elems + 255) / 256)), 256, 0, st,
@@ -1451,8 +1597,7 @@ int dkv_op_attention(const void* q, const void* k_slots, const void* v_slots, vo
   if (!q || !k_slots || !v_slots || !o || !row_off) return DKV_E_INVALID_ARG;
   if (batch < 1 || rows_per_seq_bound < 1 || seq_len < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return DKV_E_SHAPE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  static const int env_op_tc = env_int("DKV_ATTN_TC", 1);
-  if ((dtype == DKV_BF16 || dtype == DKV_F16) && head_dim == ATC_DH && env_op_tc && n_q_heads / n_kv_heads <= ATC_M) {
+  if ((dtype == DKV_BF16 || dtype == DKV_F16) && head_dim == ATC_DH && n_q_heads / n_kv_heads <= ATC_M) {
     // tensor maps for this call's buffers; the queries' row count is only known as a bound on the device,
     // so the map covers batch * bound rows (row_off never points past them)
     AttnMaps am;
@@ -1540,8 +1685,10 @@ int dkv_op_gemm_static(const void* x, const void* w, float* out, int rows, int n
   long long stride = 0;
   // part_rows bounds splits * rows, i.e. the number of [n]-float rows the scratch can hold
   const long long part_rows = max_slabs * rows;
-  rc = gemm_tc(tw, tx, n, k, rows, nullptr, scratch, part_rows, splits, nullptr, dtype == DKV_BF16, st, &s, &stride,
-               /*w_static=*/false);
+  GemmOpts o;
+  o.forced_splits = splits;
+  o.w_static = false;
+  rc = gemm_tc(tw, tx, n, k, rows, nullptr, scratch, part_rows, nullptr, dtype == DKV_BF16, st, &s, &stride, o);
   if (rc) return rc;
   // every float the reduction reads was written by the GEMM launch just above:
   // nothing in the shared scratch has to start at zero

@@ -16,6 +16,21 @@
 // units and, when tensor memory has room for two accumulators, the epilogue of
 // one unit overlaps the main loop of the next.
 //
+// Epilogues.  Every mode can scale row r of the result by a per-row factor (the
+// RMSNorm of the operand applied AFTER the product: norm(h) W^T = (h .* g) W^T / rms(h), so the
+// producer of the operand writes h .* g and the sums of squares, and this kernel divides).  Beyond
+// the plain fp32 partial sums there are fused row epilogues that need the COMPLETE sum over K and
+// a whole head or row: the CTAs that share a weight tile (its K splits) first leave their partial
+// sums in scratch (they stay in L2), count themselves on a per-tile counter, wait for the others
+// (a bounded spin: all CTAs of such a launch are resident at once, the host launches this mode
+// only when units <= SMs), and then each of them finishes a slice of the tile's rows:
+//   FUSE_RESID  h += sum; the row's sum of squares over the tile's columns; h .* gain as the
+//               next GEMM's 16-bit operand  (residual + RMSNorm around the O and down projections)
+//   FUSE_QKV    sum -> RoPE at the row's original position -> q to the compact buffer, k and v
+//               into the row's own cache slot  (Algorithm 1: the fresh K/V join the cache)
+// so the split-K reduction, the residual, the norm statistics, RoPE and the K/V scatter need no
+// kernel of their own.
+//
 // Warp roles (320 threads): warp 0 = TMA producer, warp 1 = TMEM allocation and
 // MMA issue, warps 2..9 = epilogue: two warps per TMEM lane quarter, which take
 // alternate 16-column groups of the accumulator (the epilogue of a launch with
@@ -39,6 +54,12 @@ constexpr int DEV_ERR_WAIT = 8;         // a bounded wait inside a kernel ran ou
 
 constexpr int GEMM_A_BYTES = GEMM_BM * GEMM_BK * 2;  // 16 KB of weights per 128-row half per stage
 constexpr int GEMM_MAX_STAGES = 12;
+constexpr int GEMM_BAR_BYTES = 512;      // barriers, the TMEM slot and the abort flag
+constexpr int GEMM_SCALE_BYTES = 1024;   // per-row scales of the unit's row tile (256 floats)
+
+constexpr int FUSE_NONE = 0;
+constexpr int FUSE_RESID = 1;
+constexpr int FUSE_QKV = 2;
 
 // Shared/tensor-memory plan for a row tile of `br` rows (a multiple of 16, at
 // most 256) and `halves` (1 or 2) 128-row weight halves per tile.
@@ -61,7 +82,7 @@ inline GemmTcPlan gemm_tc_plan(int br, int halves, int ctas_per_sm) {
   p.stages = budget / p.stage_bytes;
   if (p.stages > GEMM_MAX_STAGES) p.stages = GEMM_MAX_STAGES;
   if (p.stages < 2) p.stages = 2;
-  p.smem_bytes = p.stages * p.stage_bytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+  p.smem_bytes = p.stages * p.stage_bytes + 1024 /*alignment slack*/ + GEMM_BAR_BYTES + GEMM_SCALE_BYTES;
   p.ctas_per_sm = ctas_per_sm;
   return p;
 }
@@ -101,7 +122,179 @@ struct GemmTcParams {
   float* st_t;             // sum exp(l - max)(l - max)
   int w_static;            // 1: the weights were complete long before this launch, so they may be
                            // fetched before the wait on the stream predecessor
+  // per-row scale of the result: NULL = none; rs_parts > 0: rs_src is [rs_parts][rs_ld] partial sums of
+  // squares of the operand rows and the scale is rsqrt(sum / rs_d + rs_eps); rs_parts == 0: rs_src [rows]
+  // holds the ready factors
+  const float* rs_src;
+  int rs_parts;
+  long long rs_ld;
+  float rs_inv_d, rs_eps;
+  // fused row epilogue across the CTAs of a weight tile (FUSE_*); needs units <= resident CTAs
+  int fuse_mode;
+  unsigned int* tile_cnt;  // [weight tiles * row tiles] arrival counters, zero between launches
+  // FUSE_RESID
+  float* h;                // [rows][n] residual stream, updated in place
+  const float* gain;       // [n] gains of the norm that follows
+  void* xn_out;            // [rows][n] 16-bit: h .* gain
+  float* ssq_out;          // [weight tiles][ssq_ld]: each row's sum of squares over the tile's columns
+  long long ssq_ld;
+  // FUSE_QKV (n = (n_q_heads + 2 n_kv_heads) * head_dim, heads never straddle a weight tile)
+  const int32_t* act_idx;  // [rows] flattened position b * seq_len + pos of each row
+  const float2* rope_tab;  // [seq_len][head_dim / 2] (cos, sin)
+  int seq_len, n_q_heads, n_kv_heads, head_dim;
+  void* q_out;             // [rows][n_q_heads * head_dim] 16-bit
+  void* k_slots;           // [batch][n_kv_heads][seq_len][head_dim] 16-bit, this layer
+  void* v_slots;
 };
+
+__device__ __forceinline__ void named_bar_sync(int id, int n_threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint16_t to_bits16(float v, int bf16) {
+  return bf16 ? __bfloat16_as_ushort(__float2bfloat16_rn(v)) : __half_as_ushort(__float2half_rn(v));
+}
+__device__ __forceinline__ uint2 pack4_16(float a, float b, float c, float d, int bf16) {
+  uint2 o;
+  if (bf16) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    o.x = *reinterpret_cast<uint32_t*>(&lo);
+    o.y = *reinterpret_cast<uint32_t*>(&hi);
+  } else {
+    __half2 lo = __floats2half2_rn(a, b), hi = __floats2half2_rn(c, d);
+    o.x = *reinterpret_cast<uint32_t*>(&lo);
+    o.y = *reinterpret_cast<uint32_t*>(&hi);
+  }
+  return o;
+}
+
+// Second phase of the fused row epilogues, run by the 8 epilogue warps of every CTA of a weight tile
+// once all K splits of the tile have left their partial sums in scratch: this CTA finishes rows
+// [row_lo, row_hi) of the tile.  One warp per row, each lane two groups of four columns; a warp works
+// on FUSE_ROWS rows at once and requests the partials of four splits of all of them before it adds any
+// (the phase is bound by how many L2 loads are in flight, not by their number).
+constexpr int FUSE_ROWS = 2;
+
+// sums over the K splits of the float4 at element offset at[i] (i < FUSE_ROWS * 2), added onto acc[i];
+// the partials of up to five splits of all four items are requested before any is added
+constexpr int FUSE_BATCH = 5;
+__device__ __forceinline__ void sum_splits(const GemmTcParams& p, const long long (&at)[FUSE_ROWS * 2],
+                                           const bool (&on)[FUSE_ROWS * 2], float4 (&acc)[FUSE_ROWS * 2]) {
+  for (int s0 = 0; s0 < p.splits; s0 += FUSE_BATCH) {
+    float4 v[FUSE_BATCH][FUSE_ROWS * 2];
+#pragma unroll
+    for (int u = 0; u < FUSE_BATCH; ++u) {
+#pragma unroll
+      for (int i = 0; i < FUSE_ROWS * 2; ++i)
+        v[u][i] = (on[i] && s0 + u < p.splits)
+                      ? __ldcg(reinterpret_cast<const float4*>(p.out + (s0 + u) * p.split_stride + at[i]))
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < FUSE_BATCH; ++u) {
+#pragma unroll
+      for (int i = 0; i < FUSE_ROWS * 2; ++i) {
+        acc[i].x += v[u][i].x;
+        acc[i].y += v[u][i].y;
+        acc[i].z += v[u][i].z;
+        acc[i].w += v[u][i].w;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void fused_rows_resid(const GemmTcParams& p, int n0, int tile_rows, int row_lo, int row_hi,
+                                                 int ewarp, int lane) {
+  const int tile_n = n0 / tile_rows;
+  for (int rb = row_lo + ewarp * FUSE_ROWS; rb < row_hi; rb += 8 * FUSE_ROWS) {
+    long long at[FUSE_ROWS * 2];
+    bool on[FUSE_ROWS * 2];
+    float4 acc[FUSE_ROWS * 2];
+#pragma unroll
+    for (int i = 0; i < FUSE_ROWS * 2; ++i) {
+      const int r = rb + (i >> 1), n = n0 + (i & 1) * 128 + lane * 4;
+      on[i] = r < row_hi && (i & 1) * 128 < tile_rows && n < p.n;
+      at[i] = static_cast<long long>(r) * p.ldo + n;
+      acc[i] = on[i] ? __ldcg(reinterpret_cast<const float4*>(p.h + at[i])) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    sum_splits(p, at, on, acc);
+#pragma unroll
+    for (int rr = 0; rr < FUSE_ROWS; ++rr) {
+      float ss = 0.f;
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int i = rr * 2 + hf;
+        if (on[i]) {
+          const float4 a = acc[i];
+          *reinterpret_cast<float4*>(p.h + at[i]) = a;
+          ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+          const float4 g = __ldg(reinterpret_cast<const float4*>(p.gain + n0 + hf * 128 + lane * 4));
+          *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.xn_out) + at[i]) =
+              pack4_16(a.x * g.x, a.y * g.y, a.z * g.z, a.w * g.w, p.x_bf16);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      if (lane == 0 && rb + rr < row_hi) p.ssq_out[tile_n * p.ssq_ld + rb + rr] = ss;
+    }
+  }
+}
+
+// A tile of 256 columns holds 256 / head_dim whole heads and a head's rotation pairs are (i, i + head_dim/2):
+// head_dim / 8 lanes per head, each with pairs i..i+3, is exactly one warp per row (head_dim 64 or 128).
+__device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, int tile_rows, int row_lo, int row_hi,
+                                               int ewarp, int lane) {
+  const int hd = p.head_dim, half = hd >> 1;
+  const int lanes_per_head = hd >> 3;
+  const int hh = lane / lanes_per_head, i0 = (lane - hh * lanes_per_head) * 4;
+  const int col0 = n0 + hh * hd;                         // first column of this lane's head
+  const bool head_on = hh * hd < tile_rows && col0 < p.n;
+  const int head = col0 / hd;                            // q heads, then k heads, then v heads
+  const int d_q = p.n_q_heads * hd;
+  const bool is_q = head < p.n_q_heads;
+  const bool rot = head < p.n_q_heads + p.n_kv_heads;
+  const int hk = head - p.n_q_heads - (rot ? 0 : p.n_kv_heads);
+  for (int rb = row_lo + ewarp * FUSE_ROWS; rb < row_hi; rb += 8 * FUSE_ROWS) {
+    long long at[FUSE_ROWS * 2];
+    bool on[FUSE_ROWS * 2];
+    float4 acc[FUSE_ROWS * 2];
+#pragma unroll
+    for (int i = 0; i < FUSE_ROWS * 2; ++i) {
+      const int r = rb + (i >> 1);
+      on[i] = head_on && r < row_hi;
+      at[i] = static_cast<long long>(r) * p.ldo + col0 + i0 + (i & 1) * half;     // x1 group, x2 group
+      acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    sum_splits(p, at, on, acc);
+#pragma unroll
+    for (int rr = 0; rr < FUSE_ROWS; ++rr) {
+      const int r = rb + rr;
+      if (!on[rr * 2]) continue;
+      const int flat = p.act_idx[r];
+      const int b = flat / p.seq_len, pos = flat - b * p.seq_len;
+      float4 x1 = acc[rr * 2], x2 = acc[rr * 2 + 1];
+      if (rot) {
+        const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + static_cast<long long>(pos) * half + i0);
+        const float4 t0 = __ldg(tab), t1 = __ldg(tab + 1);      // (cos, sin) of i0, i0+1 | i0+2, i0+3
+        const float4 y1 = make_float4(x1.x * t0.x - x2.x * t0.y, x1.y * t0.z - x2.y * t0.w,
+                                      x1.z * t1.x - x2.z * t1.y, x1.w * t1.z - x2.w * t1.w);
+        const float4 y2 = make_float4(x2.x * t0.x + x1.x * t0.y, x2.y * t0.z + x1.y * t0.w,
+                                      x2.z * t1.x + x1.z * t1.y, x2.w * t1.z + x1.w * t1.w);
+        x1 = y1;
+        x2 = y2;
+      }
+      uint16_t* dst = is_q ? static_cast<uint16_t*>(p.q_out) + static_cast<long long>(r) * d_q + head * hd
+                           : static_cast<uint16_t*>(rot ? p.k_slots : p.v_slots) +
+                                 ((static_cast<long long>(b) * p.n_kv_heads + hk) * p.seq_len + pos) * hd;
+      *reinterpret_cast<uint2*>(dst + i0) = pack4_16(x1.x, x1.y, x1.z, x1.w, p.x_bf16);
+      *reinterpret_cast<uint2*>(dst + i0 + half) = pack4_16(x2.x, x2.y, x2.z, x2.w, p.x_bf16);
+    }
+  }
+}
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, GemmTcParams p) {
@@ -266,6 +459,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     // ------------------------------------------------------------ epilogue
     const int q = warp & 3;           // TMEM lane quarter this warp may read
     const int cs = (warp - 2) >> 2;   // which of the alternating 16-column groups this warp takes
+    const int et = threadIdx.x - 64;  // 0..255 among the epilogue threads
+    float* s_rs = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + GEMM_BAR_BYTES);   // [256] row scales
     pdl_wait();              // the row count and the output buffer belong to earlier kernels
     if (trace_on() && threadIdx.x == 64) trace_store(3, t_enter);
     int r_valid = p.r_bound;
@@ -277,6 +472,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       decode(u, n0, r0, split, kb0, n_kb);
       const int buf = j % p.n_bufs;
       const uint32_t use = static_cast<uint32_t>(j / p.n_bufs);
+      // The row scales of this unit's row tile (1 when the launch has none), computed while the MMAs run.
+      if (j > 0) named_bar_sync(1, 256);          // everyone is done with the previous unit's scales
+      {
+        float sc = 1.f;
+        const int r = r0 + et;
+        if (p.rs_src && r < r_valid) {
+          if (p.rs_parts > 0) {
+            float ss = 0.f;
+            for (int i = 0; i < p.rs_parts; ++i) ss += __ldcg(p.rs_src + i * p.rs_ld + r);
+            sc = rsqrtf(ss * p.rs_inv_d + p.rs_eps);
+          } else {
+            sc = __ldcg(p.rs_src + r);
+          }
+        }
+        s_rs[et] = sc;
+      }
+      named_bar_sync(1, 256);
       ok = mbar_wait_bounded(smem_u32(&acc_full[buf]), use & 1, abort_flag, GEMM_WAIT_CYCLES);
       if (!ok) break;
       tc_fence_after();
@@ -303,14 +515,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             if (p.x_bf16) {
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj) {
-                const float gt = __uint_as_float(vg[jj]);
-                bits[jj] = __bfloat16_as_ushort(__float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(vu[jj])));
+                const float sc = s_rs[c + jj];
+                const float gt = __uint_as_float(vg[jj]) * sc;
+                bits[jj] = __bfloat16_as_ushort(__float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * (__uint_as_float(vu[jj]) * sc)));
               }
             } else {
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj) {
-                const float gt = __uint_as_float(vg[jj]);
-                bits[jj] = __half_as_ushort(__float2half_rn(__fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(vu[jj])));
+                const float sc = s_rs[c + jj];
+                const float gt = __uint_as_float(vg[jj]) * sc;
+                bits[jj] = __half_as_ushort(__float2half_rn(__fdividef(gt, 1.f + __expf(-gt)) * (__uint_as_float(vu[jj]) * sc)));
               }
             }
             if (n_ok == 16) {
@@ -334,6 +548,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           if (n_kb > 0) {
             tmem_ld_x16(t_addr + c, v);
             tmem_ld_wait();
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) v[jj] = __float_as_uint(__uint_as_float(v[jj]) * s_rs[c + jj]);
           } else {
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) v[jj] = 0u;
@@ -399,6 +615,39 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+
+      if (p.fuse_mode != FUSE_NONE) {
+        // Cross-CTA hand-over: this CTA's partial sums are in scratch; count it on the tile's counter
+        // and wait until all K splits of the tile are there.  Then every CTA of the tile finishes its
+        // own slice of the tile's rows.  The last CTA to get past the wait resets the counter.
+        const int tile = u / p.splits;
+        unsigned int* cnt = p.tile_cnt + tile;
+        __threadfence();
+        named_bar_sync(2, 256);
+        bool fail = false;
+        if (et == 0) {
+          atomicAdd(cnt, 1u);
+          const long long t0 = clock64();
+          while (ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits)) {
+            if (*abort_flag || clock64() - t0 > GEMM_WAIT_CYCLES) {
+              fail = true;
+              *abort_flag = 1;
+              break;
+            }
+          }
+          if (!fail && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;   // everyone has passed: reset
+          __threadfence();
+        }
+        if (bar_red_or(2, 256, fail)) {
+          ok = false;
+          break;
+        }
+        const int n_rows = max(0, min(p.br, r_valid - r0));
+        const int per = (n_rows + p.splits - 1) / p.splits;
+        const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
+        if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
+        else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
+      }
     }
   }
 

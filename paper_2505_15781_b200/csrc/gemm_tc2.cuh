@@ -5,7 +5,11 @@
 // memory).  Per 32 KB of weights a CTA therefore holds br * 64 bytes of rows
 // instead of br * 128: the ring is deeper at the same shared memory and the
 // L2 -> SM traffic of the rows halves, which is what bounds the one-CTA kernel
-// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).
+// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).  Which 128 rows a CTA
+// stages for MMA h is a matter of its TMA coordinate only: plain launches take rows
+// [h*256 + rank*128, +128) so that the tile is covered in order; the SwiGLU launch takes rows
+// [rank*256 + h*128, +128) of a weight copy grouped [128 gate | 128 up] per 256 rows, so that each CTA
+// holds the gate rows (MMA 0) and the up rows (MMA 1) of the same 128 features.
 //
 // Roles per CTA (320 threads): warp 0 = TMA producer of its own half of the
 // operands, completion counted on the LEADER's barrier (cta_group::2 loads);
@@ -86,7 +90,7 @@ inline GemmTcPlan gemm_tc2_plan(int br) {
   p.tmem_cols = p.n_bufs * 2 * p.col_stride;
   p.stages = (220 * 1024) / p.stage_bytes;
   if (p.stages > GEMM_MAX_STAGES) p.stages = GEMM_MAX_STAGES;
-  p.smem_bytes = p.stages * p.stage_bytes + 1024 + 512;
+  p.smem_bytes = p.stages * p.stage_bytes + 1024 + GEMM_BAR_BYTES + GEMM_SCALE_BYTES;
   p.ctas_per_sm = 1;
   return p;
 }
@@ -187,7 +191,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         const uint32_t a_dst = smem_base + s * p.stage_bytes;
         for (int h = 0; h < 2; ++h)
           tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, (c.kb0 + c.i) * GEMM_BK,
-                                c.n0 + h * 256 + static_cast<int>(rank) * GEMM_BM, pol_w);
+                                c.n0 + (p.swiglu_out ? static_cast<int>(rank) * 256 + h * GEMM_BM
+                                                     : h * 256 + static_cast<int>(rank) * GEMM_BM), pol_w);
       };
       auto load_b = [&](const Cursor& c, int it) {
         const int s = it % STAGES;
@@ -262,6 +267,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
     // ------------------------------------------------------------ epilogue (both CTAs, own 128 lanes)
     const int q = warp & 3;
     const int cs = (warp - 2) >> 2;   // which of the alternating 16-column groups this warp takes
+    const int et = threadIdx.x - 64;  // 0..255 among the epilogue threads
+    float* s_rs = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + GEMM_BAR_BYTES);   // [256] row scales
     pdl_wait();
     int r_valid = p.r_bound;
     if (p.r_dev) r_valid = min(r_valid, *p.r_dev);
@@ -272,6 +279,23 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
       decode(u, n0, r0, split, kb0, n_kb);
       const int buf = j % p.n_bufs;
       const uint32_t use = static_cast<uint32_t>(j / p.n_bufs);
+      // the row scales of this unit's row tile (1 when the launch has none), computed while the MMAs run
+      if (j > 0) named_bar_sync(1, 256);
+      {
+        float sc = 1.f;
+        const int r = r0 + et;
+        if (p.rs_src && r < r_valid) {
+          if (p.rs_parts > 0) {
+            float ss = 0.f;
+            for (int i = 0; i < p.rs_parts; ++i) ss += __ldcg(p.rs_src + i * p.rs_ld + r);
+            sc = rsqrtf(ss * p.rs_inv_d + p.rs_eps);
+          } else {
+            sc = __ldcg(p.rs_src + r);
+          }
+        }
+        s_rs[et] = sc;
+      }
+      named_bar_sync(1, 256);
       ok = mbar_wait_bounded(smem_u32(&acc_full[buf]), use & 1, abort_flag, GEMM_WAIT_CYCLES);
       if (!ok) break;
       tc_fence_after();
@@ -279,8 +303,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
       const int row_in_tile = static_cast<int>(rank) * GEMM_BM + q * 32 + lane;   // + h * 256
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(buf * 2 * p.col_stride);
       if (p.swiglu_out) {
-        // the gate/up copy is regrouped [256 gate rows | 256 up rows] per pair tile: gate and up of
-        // feature jf are lane `row_in_tile` of the tile's two accumulators
+        // the gate/up copy is grouped [128 gate rows | 128 up rows] per 256 rows and this CTA staged the
+        // gate rows (MMA 0) and the up rows (MMA 1) of features (n0 / 2) + rank * 128 + [0, 128)
         const int jf = (n0 >> 1) + row_in_tile;
         for (int c = cs * 16; c < p.br; c += 32) {
           if (r0 + c >= r_valid) break;
@@ -297,14 +321,16 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
             if (p.x_bf16) {
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj) {
-                const float gt = __uint_as_float(vg[jj]);
-                bits[jj] = __bfloat16_as_ushort(__float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(vu[jj])));
+                const float sc = s_rs[c + jj];
+                const float gt = __uint_as_float(vg[jj]) * sc;
+                bits[jj] = __bfloat16_as_ushort(__float2bfloat16_rn(__fdividef(gt, 1.f + __expf(-gt)) * (__uint_as_float(vu[jj]) * sc)));
               }
             } else {
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj) {
-                const float gt = __uint_as_float(vg[jj]);
-                bits[jj] = __half_as_ushort(__float2half_rn(__fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(vu[jj])));
+                const float sc = s_rs[c + jj];
+                const float gt = __uint_as_float(vg[jj]) * sc;
+                bits[jj] = __half_as_ushort(__float2half_rn(__fdividef(gt, 1.f + __expf(-gt)) * (__uint_as_float(vu[jj]) * sc)));
               }
             }
             if (n_ok == 16) {
@@ -327,6 +353,8 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
           if (n_kb > 0) {
             tmem_ld_x16(t_addr + c, v);
             tmem_ld_wait();
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) v[jj] = __float_as_uint(__uint_as_float(v[jj]) * s_rs[c + jj]);
           } else {
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) v[jj] = 0u;

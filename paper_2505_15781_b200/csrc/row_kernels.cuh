@@ -83,12 +83,49 @@ __global__ void k_rope_table(float2* tab, int seq_len, int half, double theta) {
   tab[idx] = make_float2(static_cast<float>(cos(a)), static_cast<float>(sin(a)));
 }
 
-// h[r] = E[tokens[act_idx[r]]];  xn[r] = RMSNorm(h[r]) * gain   (one CTA per row)
+// 8 consecutive elements of an embedding row as floats (16-byte loads)
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  const float4 a = __ldg(reinterpret_cast<const float4*>(p)), b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+  v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 u = __ldg(reinterpret_cast<const uint4*>(p));
+  const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float2 f = __bfloat1622float2(b[j]);
+    v[2 * j] = f.x;
+    v[2 * j + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+  reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+  reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
+  uint4 o;
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) h[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+  *reinterpret_cast<uint4*>(p) = o;
+}
+__device__ __forceinline__ void store8(__half* p, const float (&v)[8]) {
+  uint4 o;
+  __half2* h = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) h[j] = __floats2half2_rn(v[2 * j], v[2 * j + 1]);
+  *reinterpret_cast<uint4*>(p) = o;
+}
+
+// h[r] = E[tokens[act_idx[r]]] and the operand of the first QKV projection (one CTA per row, 16-byte
+// accesses, d a multiple of 8).  ssq == NULL: xn[r] = RMSNorm(h[r]) * gain.  ssq != NULL: xn[r] =
+// h[r] .* gain and ssq[r] = sum h[r]^2; the GEMM that reads xn divides by the RMS in its epilogue.
 template <typename TW, typename T>
 __global__ void __launch_bounds__(256)
 k_embed_norm(const TW* __restrict__ embed, const int32_t* __restrict__ tokens, const int32_t* __restrict__ act_idx,
              const int* __restrict__ r_dev, const float* __restrict__ gain, float eps, int d, float* __restrict__ h,
-             T* __restrict__ xn) {
+             T* __restrict__ xn, float* __restrict__ ssq) {
   __shared__ float s8[8];
   pdl_enter(2);
   const int r = blockIdx.x;
@@ -96,16 +133,55 @@ k_embed_norm(const TW* __restrict__ embed, const int32_t* __restrict__ tokens, c
   const int tok = tokens[act_idx[r]];
   const TW* e = embed + static_cast<long long>(tok) * d;
   float* hr = h + static_cast<long long>(r) * d;
+  T* xr = xn + static_cast<long long>(r) * d;
+  constexpr int KEEP = 4;                     // row pieces of 2048 elements kept in registers (d <= 8192)
+  float v[KEEP][8];
   float ss = 0.f;
-  for (int c = threadIdx.x; c < d; c += 256) {
-    const float v = to_f32(e[c]);
-    hr[c] = v;
-    ss += v * v;
+  auto first_pass = [&](int c, float (&t)[8]) {
+    load8(e + c, t);
+    store8(hr + c, t);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) ss += t[j] * t[j];
+    if (ssq) {                                 // h .* gain needs no statistic of the row
+      float g[8], o[8];
+      load8(gain + c, g);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) o[j] = t[j] * g[j];
+      store8(xr + c, o);
+    }
+  };
+#pragma unroll
+  for (int i = 0; i < KEEP; ++i) {
+    const int c = threadIdx.x * 8 + i * 2048;
+    if (c < d) first_pass(c, v[i]);
+  }
+  for (int c = threadIdx.x * 8 + KEEP * 2048; c < d; c += 2048) {
+    float t[8];
+    first_pass(c, t);
   }
   ss = block_sum_256(ss, s8);
+  if (ssq) {
+    if (threadIdx.x == 0) ssq[r] = ss;
+    return;
+  }
   const float inv = rsqrtf(ss / static_cast<float>(d) + eps);
-  T* xr = xn + static_cast<long long>(r) * d;
-  for (int c = threadIdx.x; c < d; c += 256) xr[c] = from_f32<T>(hr[c] * inv * gain[c]);
+  auto second_pass = [&](int c, float (&t)[8]) {
+    float g[8];
+    load8(gain + c, g);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) t[j] = t[j] * inv * g[j];
+    store8(xr + c, t);
+  };
+#pragma unroll
+  for (int i = 0; i < KEEP; ++i) {
+    const int c = threadIdx.x * 8 + i * 2048;
+    if (c < d) second_pass(c, v[i]);
+  }
+  for (int c = threadIdx.x * 8 + KEEP * 2048; c < d; c += 2048) {
+    float t[8];
+    load8(hr + c, t);
+    second_pass(c, t);
+  }
 }
 
 __device__ __forceinline__ void store4(float* p, float a, float b, float c, float d) {
@@ -135,11 +211,12 @@ __device__ __forceinline__ void add4(float4& a, const float4 b) {
 // h[r] += sum_s part[s][r];  xn[r] = RMSNorm(h[r]) * gain     (one CTA per row;
 // float4 accesses, d a multiple of 4; up to 4 x 256 float4 per pass are kept in
 // flight per thread block so the split-K partials are read with wide parallelism)
+// ssq != NULL: xn[r] = h[r] .* gain and ssq[r] = sum h[r]^2 instead (the consuming GEMM divides by the RMS).
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_resid_norm(float* __restrict__ h, const float* __restrict__ part, int splits, long long split_stride,
              const int* __restrict__ r_dev, const float* __restrict__ gain, float eps, int d,
-             T* __restrict__ xn) {
+             T* __restrict__ xn, float* __restrict__ ssq) {
   __shared__ float s8[8];
   pdl_enter(7);
   const int r = blockIdx.x;
@@ -185,7 +262,11 @@ k_resid_norm(float* __restrict__ h, const float* __restrict__ part, int splits, 
     }
   }
   ss = block_sum_256(ss, s8);
-  const float inv = rsqrtf(ss / static_cast<float>(d) + eps);
+  float inv = rsqrtf(ss / static_cast<float>(d) + eps);
+  if (ssq) {
+    if (threadIdx.x == 0) ssq[r] = ss;
+    inv = 1.f;
+  }
   T* xr = xn + static_cast<long long>(r) * d;
   if (nvec <= 4 * 256) {
     // one pass held the whole row: normalise from registers instead of reading h back
@@ -278,17 +359,27 @@ k_swiglu(const float* __restrict__ part, int splits, long long split_stride, con
   }
 }
 
-// xh[i] = xn[head_row[i]] for i < n_head (device count)
+// xh[i] = xn[head_row[i]] for i < n_head (device count), 16-byte copies (d a multiple of 8 elements of
+// 2 bytes, or of 4 floats).  With ssq != NULL (xn holds h .* gain) also head_rs[i] = the row's
+// 1 / RMS from its ssq_parts partial sums of squares [ssq_parts][ssq_ld].
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_head_gather(const T* __restrict__ xn, const int32_t* __restrict__ head_row, const int* __restrict__ n_head_dev,
-              int d, T* __restrict__ xh) {
+              int d, T* __restrict__ xh, const float* __restrict__ ssq, int ssq_parts, long long ssq_ld, float eps,
+              float* __restrict__ head_rs) {
   pdl_enter(11);
   const int i = blockIdx.x;
   if (i >= *n_head_dev) return;
-  const T* src = xn + static_cast<long long>(head_row[i]) * d;
-  T* dst = xh + static_cast<long long>(i) * d;
-  for (int c = threadIdx.x; c < d; c += 256) dst[c] = src[c];
+  const int row = head_row[i];
+  const uint4* src = reinterpret_cast<const uint4*>(xn + static_cast<long long>(row) * d);
+  uint4* dst = reinterpret_cast<uint4*>(xh + static_cast<long long>(i) * d);
+  const int n16 = d * static_cast<int>(sizeof(T)) / 16;
+  for (int c = threadIdx.x; c < n16; c += 256) dst[c] = src[c];
+  if (ssq && threadIdx.x == 0) {
+    float ss = 0.f;
+    for (int t = 0; t < ssq_parts; ++t) ss += ssq[t * ssq_ld + row];
+    head_rs[i] = rsqrtf(ss / static_cast<float>(d) + eps);
+  }
 }
 
 // Sum split-K partials of the head GEMM into the logits buffer (only needed when splits > 1

@@ -121,6 +121,23 @@ def test_policies_bf16_batch2_gqa(pol, k):
     run_forced(GQA, True, 2, 11, 16, k, pol, None, seed=2, with_order=pol.kind == O.POLICY_GREEDY)
 
 
+MEDIUM_128 = synth.ModelShape(2, 1024, 8, 2, 128, 1536, 2000, 1999)    # K splits of 4-6, CTA-pair gate/up launch
+MEDIUM_64 = synth.ModelShape(2, 768, 12, 4, 64, 1024, 1500, 1499)      # head_dim 64: four heads per weight tile
+
+
+@pytest.mark.parametrize("fuse", [1, 0])
+@pytest.mark.parametrize("ms,pol,k", [(MEDIUM_128, O.Policy(O.POLICY_DECODE, 3), 2),
+                                      (MEDIUM_64, O.Policy(O.POLICY_PD, 2), 3),
+                                      (MEDIUM_128, O.Policy(O.POLICY_PREFILL, isolated_prefill=True), 2)])
+def test_medium_widths_split_k_with_and_without_fused_tails(ms, pol, k, fuse, monkeypatch):
+    """Widths at which the projections run with several K splits: with the fused tails (the CTAs of a
+    weight tile reduce the splits and apply residual / norm statistics / RoPE / slot scatter themselves)
+    and with the switch off (partials to scratch, row kernels), against the oracle, both head paths."""
+    monkeypatch.setenv("DKV_FUSE_TAILS", str(fuse))
+    worst = run_forced(ms, True, 2, 37, 12 * k, k, pol, 6 * k, seed=5)
+    assert worst < BF16_TOL_SIGMA
+
+
 def free_run(ms, bf16, batch, P, G, k, pol, block, seed=0, host=False):
     W, model = U.build_pair(ms, seed, bf16)
     prompts = synth.make_prompt(batch, P, min(1000, ms.vocab - 1), seed)
