@@ -40,6 +40,11 @@ WORKLOADS = {
                        window=0),
     "llada8b_greedy": dict(shape="llada", batch=1, prompt=128, gen=1024, block=1024, k=1, policy="greedy",
                            interval=2, window=4),
+    # the comparison runs of the same shape (prompt 128, generation 1024, no blocks, one token per step)
+    "llada8b_long_nocache": dict(shape="llada", batch=1, prompt=128, gen=1024, block=1024, k=1, policy="none",
+                                 interval=0, window=0),
+    "llada8b_long_decode": dict(shape="llada", batch=1, prompt=128, gen=1024, block=1024, k=1, policy="decode",
+                                interval=8, window=0),
     # depth-truncated copy of the default workload (a few GB on the device): the case ncu captures
     "llada8b_decode_2layers": dict(shape="llada", layers=2, batch=1, prompt=256, gen=256, block=32, k=1,
                                    policy="decode", interval=8, window=0),
@@ -48,9 +53,11 @@ WORKLOADS = {
 }
 
 
-# DRAM traffic (read + write) per launch of k_gemm_tc from the ncu capture summarised in
-# profiles/k_gemm_tc_llada8b_decode_2layers.md (254 active rows; per launch, independent of depth)
+# DRAM traffic (read + write) per launch of the projection GEMMs: a RECORDED constant from the ncu capture
+# summarised in profiles/k_gemm_tc_llada8b_decode_2layers.md (254 active rows; per launch, independent of
+# depth), not measured by this run.
 NCU_GEMM_TRAFFIC = {"gemm_qkv": 106.3e6, "gemm_o": 36.2e6, "gemm_gateup": 207.5e6, "gemm_down": 110.4e6}
+NCU_GEMM_TRAFFIC_SOURCE = "ncu capture summarised in profiles/k_gemm_tc_llada8b_decode_2layers.md (recorded constant)"
 
 
 def peaks():
@@ -124,6 +131,19 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def step_costs(ms, wl, rows, full_rows):
+    """Algorithmic cost of one step with `rows` active rows in total (all sequences) whose queries attend
+    `full_rows` slots per sequence: weight bytes (every projection matrix and the head once: the per-step
+    figure of the hot-path table), K/V slot bytes, flops."""
+    d, L = ms.d_model, full_rows
+    w_bytes = 2.0 * (ms.n_layers * ms.params_per_layer() + ms.vocab * d)
+    kv_bytes = 2.0 * 2 * wl["batch"] * L * ms.d_kv * ms.n_layers
+    head_rows = min(wl["block"], wl["gen"]) * wl["batch"]
+    flops = 2.0 * rows * ms.n_layers * ms.params_per_layer() + 4.0 * rows * L * ms.d_q * ms.n_layers + \
+        2.0 * head_rows * ms.vocab * d
+    return w_bytes, kv_bytes, flops
+
+
 def shape_of(wl):
     from paper_2505_15781_b200 import synth
     ms = {"llada": synth.llada_shape, "dream": synth.dream_shape, "tiny": synth.tiny_shape}[wl["shape"]]()
@@ -137,7 +157,9 @@ def shape_of(wl):
 class Job:
     """One replica of the workload on the current device."""
 
-    def __init__(self, wl, seed=0):
+    def __init__(self, wl, seed=0, order=None, model=None):
+        """order: [T, batch, k] device tensor of positions to unmask (a recorded or predefined order; required
+        for Greedy, optional replay for the other policies).  model: reuse a built model of the same shape."""
         import torch
         from paper_2505_15781_b200 import binding as B
         from paper_2505_15781_b200 import synth
@@ -146,9 +168,11 @@ class Job:
         self.ms = ms
         bf16 = wl["shape"] != "tiny"
         self.dtype = "bf16" if bf16 else "f32"
-        w = synth.make_weights(ms, seed, "bfloat16" if bf16 else "float32", "cuda")
-        self.model = B.dkv_model_create(ms, w, B.DKV_BF16 if bf16 else B.DKV_F32)
-        del w
+        if model is None:
+            w = synth.make_weights(ms, seed, "bfloat16" if bf16 else "float32", "cuda")
+            model = B.dkv_model_create(ms, w, B.DKV_BF16 if bf16 else B.DKV_F32)
+            del w
+        self.model = model
         kind = {"decode": B.DKV_POLICY_DECODE, "none": B.DKV_POLICY_NONE, "pd": B.DKV_POLICY_PD,
                 "prefill": B.DKV_POLICY_PREFILL, "greedy": B.DKV_POLICY_GREEDY}[wl["policy"]]
         self.policy = B.make_policy(kind, wl["interval"], 1, wl["window"], B.DKV_CENTER_PREV,
@@ -160,8 +184,8 @@ class Job:
         x0, m0 = synth.initial_state(prompts, self.G, ms.mask_id)
         self.x0, self.m0 = torch.from_numpy(x0).cuda(), torch.from_numpy(m0).cuda()
         self.x, self.m = self.x0.clone(), self.m0.clone()
-        self.order = None
-        if wl["policy"] == "greedy":
+        self.order = order
+        if wl["policy"] == "greedy" and order is None:
             self.order = torch.from_numpy(synth.random_order(self.batch, self.P, self.G, self.k, seed)).cuda()
         need = B.dkv_cache_bytes(self.model, self.batch, self.L, self.policy)
         self.arena = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
@@ -180,6 +204,15 @@ class Job:
     def total_launches(self):
         return self.launches + (self.B.dkv_get_stats(self.cache).kernel_launches if self.cache else 0)
 
+    def record_order(self):
+        """One whole generation; returns the positions it unmasked, [T, batch, k] on the device."""
+        self.restart()
+        chosen = self.torch.full((self.T, self.batch, self.k), -1, dtype=self.torch.int32, device="cuda")
+        self.B.dkv_generate(self.cache, self.x, self.m, self.order, self.k, self.wl["block"], 0, chosen)
+        self.torch.cuda.synchronize()
+        self.pos = self.T
+        return chosen
+
     def run_steps(self, n, profile_cb=None):
         """n consecutive denoising steps on the device (generations wrap)."""
         done = 0
@@ -197,6 +230,19 @@ class Job:
                     profile_cb(self.pos)
                     self.pos += 1
                     done += 1
+
+    def active_rows(self, s):
+        """Rows one sequence recomputes at 0-based step s (the host-side bound the library is given)."""
+        pol = self.wl["policy"]
+        if pol == "none" or s == 0:
+            return self.L
+        if pol == "prefill" or (pol == "pd" and self.is_refresh(s)):
+            return self.G
+        if self.is_refresh(s):
+            return self.L
+        if pol == "greedy":
+            return min(self.L, self.k * (self.wl["window"] + 2))
+        return min(self.L, self.G - s * self.k + self.k)
 
     def is_refresh(self, s):
         pol, N = self.wl["policy"], self.wl["interval"]
@@ -279,7 +325,7 @@ def run_ours(args, rank, world):
 
     # ------------------------------------------------ per-kernel pass (events around every launch)
     pk = peaks()
-    roofline, roofline_tensor, classes = None, None, {}
+    roofline, roofline_tensor, roofline_attn, classes = None, None, None, {}
     if rank == 0:
         job.restart()
         job.run_steps(first)
@@ -293,15 +339,23 @@ def run_ours(args, rank, world):
                 a = bucket.setdefault(e["name"], dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
                 for key in ("launches", "ms", "bytes", "flops"):
                     a[key] += e[key]
-        job.run_steps(min(K, job.T), profile_cb=cb)
+        n_prof = min(K, job.T)
+        job.run_steps(n_prof, profile_cb=cb)
         B.dkv_profile_enable(job.cache, False)
+        ms_shape = job.ms
+
+        # weight bytes of one launch of each GEMM class (the hot-path table's per-unit figure: 2 K N)
+        d_, f_ = ms_shape.d_model, ms_shape.d_ffn
+        w_bytes = {"gemm_qkv": 2.0 * (ms_shape.d_q + 2 * ms_shape.d_kv) * d_, "gemm_o": 2.0 * d_ * ms_shape.d_q,
+                   "gemm_gateup": 2.0 * 2 * f_ * d_, "gemm_down": 2.0 * d_ * f_, "gemm_head": 2.0 * ms_shape.vocab * d_}
 
         def gemm_sum(bucket):
-            tot = dict(launches=0, ms=0.0, bytes=0.0, flops=0.0)
+            tot = dict(launches=0, ms=0.0, bytes=0.0, flops=0.0, weight_bytes=0.0)
             for name, a in bucket.items():
                 if name.startswith("gemm_"):
-                    for key in tot:
+                    for key in ("launches", "ms", "bytes", "flops"):
                         tot[key] += a[key]
+                    tot["weight_bytes"] += a["launches"] * w_bytes[name]
             return tot
         gc, gr = gemm_sum(agg["cached"]), gemm_sum(agg["refresh"])
         traffic = None
@@ -310,34 +364,55 @@ def run_ours(args, rank, world):
             if cls:
                 traffic = sum(NCU_GEMM_TRAFFIC[n] * c for n, c in cls) / sum(c for _, c in cls)
         if gc["launches"]:
-            ach = gc["bytes"] / (gc["ms"] * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "k_gemm_tc / k_gemm_tc2 (tcgen05 projection GEMMs), launches of the cached steps",
+            ach = gc["weight_bytes"] / (gc["ms"] * 1e-3) / 1e9
+            ach_full = gc["bytes"] / (gc["ms"] * 1e-3) / 1e9
+            roofline = {"bound": "hbm",
+                        "kernel": "k_gemm_tc / k_gemm_tc2 (tcgen05 projection GEMMs with their fused row tails: split-K "
+                                  "reduction, residual, norm statistics, RoPE, K/V scatter, SwiGLU, head statistics), "
+                                  "launches of the cached steps",
                         "achieved": ach, "peak": pk["hbm"], "unit": "GB/s", "frac": ach / pk["hbm"],
+                        "bytes": "weights only (2 K N per launch)",
                         "peak_source": f"of {pk['src']}", "peak_nominal": 7700.0, "frac_of_nominal": ach / 7700.0,
-                        "traffic": traffic,
-                        "traffic_note": "DRAM bytes per launch, ncu capture at 254 rows, mean over the layer's "
-                                        "four GEMM shapes (head launches not captured)",
+                        "with_rows_and_outputs": {"achieved": ach_full, "frac": ach_full / pk["hbm"],
+                                                  "bytes": "weights + row operands + results"},
+                        "traffic": traffic, "traffic_source": NCU_GEMM_TRAFFIC_SOURCE,
                         "launches": gc["launches"], "avg_launch_us": gc["ms"] * 1e3 / gc["launches"],
-                        "algorithmic_bytes_per_launch": gc["bytes"] / gc["launches"]}
+                        "algorithmic_bytes_per_launch": gc["weight_bytes"] / gc["launches"]}
         if gr["launches"]:
             ach = gr["flops"] / (gr["ms"] * 1e-3) / 1e12
-            roofline_tensor = {"bound": "tensor", "kernel": "k_gemm_tc, launches of the refresh steps",
-                               "achieved": ach, "peak": pk["tf_sust"], "unit": "TFLOP/s", "frac": ach / pk["tf_sust"],
-                               "peak_source": f"of {pk['src']} (sustained)", "peak_nominal": 2250.0,
-                               "frac_of_nominal": ach / 2250.0, "launches": gr["launches"],
+            roofline_tensor = {"bound": "tensor", "kernel": "k_gemm_tc / k_gemm_tc2, launches of the refresh steps "
+                                                            "(each timed alone between events: burst peak)",
+                               "achieved": ach, "peak": pk["tf_burst"], "unit": "TFLOP/s", "frac": ach / pk["tf_burst"],
+                               "peak_source": f"of {pk['src']} (burst)", "frac_of_sustained": ach / pk["tf_sust"],
+                               "peak_nominal": 2250.0, "frac_of_nominal": ach / 2250.0, "launches": gr["launches"],
                                "avg_launch_us": gr["ms"] * 1e3 / gr["launches"]}
             if roofline is None:
                 roofline = dict(roofline_tensor, traffic=None)
-        # The events of the per-kernel pass serialise the launches, so a GEMM there pays its whole ramp
-        # (no dependent-launch overlap, no weight tiles fetched ahead).  Secondary figure: the GEMMs'
-        # SHARE of that pass applied to the duration of the timed region itself.
-        prof_total = sum(a["ms"] for bucket in agg.values() for a in bucket.values())
-        n_prof = min(K, job.T)
-        if roofline and gc["launches"] and prof_total > 0:
-            in_step_ms = ms * (n_prof / K) * (gc["ms"] / prof_total)
-            roofline["in_step"] = {"achieved": gc["bytes"] / (in_step_ms * 1e-3) / 1e9, "unit": "GB/s",
-                                   "frac": gc["bytes"] / (in_step_ms * 1e-3) / 1e9 / pk["hbm"],
-                                   "how": "algorithmic bytes / (timed region x the launches' share of the per-kernel pass)"}
+        # attention against both rooflines, from the same event pass (all steps)
+        att = dict(launches=0, ms=0.0, bytes=0.0, flops=0.0)
+        for bucket in agg.values():
+            if "attention" in bucket:
+                for key in att:
+                    att[key] += bucket["attention"][key]
+        if att["launches"]:
+            tf = att["flops"] / (att["ms"] * 1e-3) / 1e12
+            gb = att["bytes"] / (att["ms"] * 1e-3) / 1e9
+            roofline_attn = {"kernel": "k_attn_tc (tcgen05 attention over the slot cache)", "launches": att["launches"],
+                             "avg_launch_us": att["ms"] * 1e3 / att["launches"], "TFLOP/s": tf,
+                             "frac_of_tensor_peak": tf / pk["tf_burst"], "GB/s": gb, "frac_of_hbm_peak": gb / pk["hbm"],
+                             "note": "launches of this size are latency-bound (few CTAs, few slot tiles each)"}
+        # Whole-window figure: roofline time of the timed steps (each step the slower of its flops at the
+        # sustained tensor peak and its weight + K/V bytes at the HBM peak) over the measured time.
+        t_roof = 0.0
+        for s_i in range(first, first + K):
+            si = s_i % job.T
+            rows = job.batch * job.active_rows(si)
+            wb, kvb, fl = step_costs(ms_shape, wl, rows, job.L)
+            t_roof += max(fl / (pk["tf_sust"] * 1e12), (wb + kvb) / (pk["hbm"] * 1e9))
+        if roofline is not None:
+            roofline["whole_window"] = {"roofline_ms": t_roof * 1e3, "measured_ms": ms, "frac": t_roof * 1e3 / ms,
+                                        "how": "sum over the timed steps of max(flops / sustained tensor peak, "
+                                               "(weight + K/V bytes) / HBM peak), over the device time of the region"}
         for bname, bucket in agg.items():
             tot = sum(a["ms"] for a in bucket.values()) or 1.0
             classes[bname] = {n: {"launches": a["launches"], "ms": round(a["ms"], 3), "share": round(a["ms"] / tot, 4)}
@@ -345,17 +420,21 @@ def run_ours(args, rank, world):
 
     out = None
     if rank == 0:
+        st = B.dkv_get_stats(job.cache)
         out = {
             "metric": "generated tokens/s (dKV-Cache denoising steps, whole hot path)",
             "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": job.dtype, "data": "synthetic",
-            "config": {"workload": args.workload, **{k: v for k, v in wl.items()},
-                       "window": f"steps {first}..{first + K - 1} of the {job.T}-step generation",
-                       "l2": "inputs larger than L2: every step streams all weights (16 GB) once",
-                       "replicas": "independent replica per GPU, no collective on the data path"},
+            "dtype": "bf16 weights as fp16, fp16 operands, fp32 accumulate" if job.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": args.workload, **{k: v for k, v in wl.items()}},
+            "timed_steps": f"steps {first}..{first + K - 1} of the {job.T}-step generation",
+            "l2": "inputs larger than L2: every step streams all weights (16 GB) once",
+            "replicas": "independent replica per GPU, no collective on the data path",
+            "memory": {"arena_bytes": int(job.arena.numel()), "kv_slot_bytes": int(st.cache_bytes)},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": status,
-            "roofline": roofline, "roofline_refresh_steps": roofline_tensor, "kernel_classes": classes,
+            "roofline": roofline, "roofline_refresh_steps": roofline_tensor, "roofline_attention": roofline_attn,
+            "kernel_classes": classes,
         }
     if world > 1:
         dist.barrier()
@@ -430,6 +509,88 @@ def run_reference(args, rank, world):
                              "sample": f"first {n} of {K} steps, one sequence; per step a 1-layer and a 0-layer model "
                                        f"are timed and the layer time scaled to full depth (extrapolated)"},
             "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def timed_generation_steps(job, steps):
+    """Device time of `steps` consecutive steps from the middle of a generation (all of it when steps >= T)."""
+    import torch
+    steps = min(steps, job.T)
+    first = (job.T - steps) // 2
+    job.run_steps(3)
+    job.restart()
+    job.run_steps(first)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    job.run_steps(steps)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1), steps, first
+
+
+def run_order_comparison(args):
+    """The long-generation comparison (prompt 128, generation 1024, no blocks, one token per step): the
+    no-cache run picks its positions by confidence; that order is recorded and REPLAYED by dKV-Cache-Decode
+    (refresh every 8 steps) and dKV-Cache-Greedy (window 4, refresh every 2 / every 8 / never), so that all
+    runs traverse one decoding order (Sec. 3.4: Greedy needs the position before the forward pass).
+    One JSON line per run; tokens/s over a whole generation unless --steps is smaller."""
+    import torch
+    from paper_2505_15781_b200 import binding as B
+    torch.cuda.set_device(0)
+    base = WORKLOADS["llada8b_long_nocache"]
+    ref = Job(base)
+    order = ref.record_order()
+    rows = []
+    for name, pol, interval, window in (("no-cache", "none", 0, 0), ("decode N=8", "decode", 8, 0),
+                                        ("greedy N=2 w=4", "greedy", 2, 4), ("greedy N=8 w=4", "greedy", 8, 4),
+                                        ("greedy no refresh w=4", "greedy", 0, 4)):
+        wl = dict(base, policy=pol, interval=interval, window=window)
+        job = Job(wl, order=order, model=ref.model)
+        ms, steps, first = timed_generation_steps(job, args.steps)
+        st = B.dkv_get_stats(job.cache)
+        assert B.dkv_status(job.cache) == 0
+        row = {"sweep": "order_comparison", "run": name, "prompt": wl["prompt"], "gen": wl["gen"], "steps": steps,
+               "first_step": first, "order": "recorded from the no-cache confidence run, replayed",
+               "tokens_per_s": steps * job.k * job.batch / (ms * 1e-3), "ms_per_step": ms / steps,
+               "cache_ratio": st.cache_ratio, "kv_slot_bytes": int(st.cache_bytes), "arena_bytes": int(job.arena.numel())}
+        rows.append(row)
+        row["speedup_vs_nocache"] = row["tokens_per_s"] / rows[0]["tokens_per_s"]
+        print(json.dumps(row), flush=True)
+        del job
+        torch.cuda.empty_cache()
+
+
+def run_length_sweep(args):
+    """Speed and memory against decode length and prefill length (the paper's memory-and-speed study,
+    Sec. 4.3): generation length x prompt length for no-cache, Decode N=8, Greedy N=2 and N=8 (window 4,
+    seeded random order), LLaDA-8B-shaped, batch 1, one token per step.  Each point times --steps steps
+    from the middle of its generation.  One JSON line per point."""
+    import torch
+    from paper_2505_15781_b200 import binding as B
+    from paper_2505_15781_b200 import synth
+    torch.cuda.set_device(0)
+    ms_shape = synth.llada_shape()
+    w = synth.make_weights(ms_shape, 0, "bfloat16", "cuda")
+    model = B.dkv_model_create(ms_shape, w, B.DKV_BF16)
+    del w
+    for gen in [int(v) for v in args.sweep_gens.split(",")]:
+        for prompt in [int(v) for v in args.sweep_prompts.split(",")]:
+            row = {"sweep": "length", "gen": gen, "prompt": prompt}
+            for name, pol, interval, window in (("none", "none", 0, 0), ("decode8", "decode", 8, 0),
+                                                ("greedy2", "greedy", 2, 4), ("greedy8", "greedy", 8, 4)):
+                wl = dict(shape="llada", batch=1, prompt=prompt, gen=gen, block=gen, k=1, policy=pol,
+                          interval=interval, window=window)
+                job = Job(wl, model=model)
+                ms, steps, first = timed_generation_steps(job, args.steps)
+                st = B.dkv_get_stats(job.cache)
+                assert B.dkv_status(job.cache) == 0
+                row[name] = {"tokens_per_s": steps / (ms * 1e-3), "ms_per_step": ms / steps,
+                             "kv_slot_gb": st.cache_bytes / 1e9, "arena_gb": job.arena.numel() / 1e9}
+                del job
+                torch.cuda.empty_cache()
+            for name in ("decode8", "greedy2", "greedy8"):
+                row[name]["speedup"] = row[name]["tokens_per_s"] / row["none"]["tokens_per_s"]
+            print(json.dumps(row), flush=True)
 
 
 def run_batch_sweep(args):
@@ -586,7 +747,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b_decode", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", default="", choices=["", "batch", "layer", "attention"])
+    ap.add_argument("--sweep", default="", choices=["", "batch", "layer", "attention", "order", "length"])
+    ap.add_argument("--sweep-gens", default="128,256,512,1024")
+    ap.add_argument("--sweep-prompts", default="0,128,512,2048")
     ap.add_argument("--attn-cases", default="254x512x1x32x32,512x512x1x32x32,1024x1024x8x32x32,4096x4096x1x32x32,"
                                             "8192x8192x1x32x32,1024x8192x1x32x32,1x8192x32x32x32,8x1152x1x32x32,768x768x4x28x4",
                     help="rows x slots x batch x query heads x KV heads, comma separated")
@@ -602,6 +765,13 @@ def main():
     if args.sweep == "attention":
         args.steps = min(args.steps, 10)
         run_attention_sweep(args)
+        return
+    if args.sweep == "order":
+        run_order_comparison(args)
+        return
+    if args.sweep == "length":
+        args.steps = min(args.steps, 64)
+        run_length_sweep(args)
         return
     if args.sweep == "layer":
         args.sweep_batches = args.sweep_batches or "1,8,32"

@@ -28,7 +28,13 @@
  *    stay within 2e-2 sigma of an exact evaluation) or DKV_BF16 (fp32's
  *    exponent range, 8-bit significand).
  *  - Positions are 0-based; step numbers t are 1-based as in the paper.
- *  - A handle is used from one host thread at a time.
+ *  - A handle is used from one host thread at a time.  A handle argument that
+ *    is not a live handle (never created, already destroyed, or a cache whose
+ *    model was destroyed) yields DKV_E_STATE; nothing is read through it.
+ *  - The kernels of this library size themselves to the whole GPU, and in some
+ *    launches the thread blocks of one launch wait for each other (bounded
+ *    waits).  Launches of the library on ONE device must therefore not overlap:
+ *    drive a device from one stream at a time.
  *  - Device-side problems (a row bound that was exceeded, fewer candidates
  *    than k, a wait inside a kernel that ran out) set a sticky status word
  *    that dkv_status() reads; kernels never trap.
@@ -204,8 +210,9 @@ int dkv_cache_destroy(dkv_cache* cache);
  *                                 stride = vocab; it must hold batch *
  *                                 max_head_rows rows
  * Updates the cache slots of A_t, the provenance stamps, the stored previous
- * mask and the step / refresh counters.  Errors: INVALID_ARG, STATE (cache
- * not initialised), SHAPE (k > max_k, cand range outside the sequence). */
+ * mask and the step / refresh counters.  Errors: INVALID_ARG, STATE (not a
+ * live handle), SHAPE (k > max_k, cand range outside the sequence; GREEDY: k
+ * differs from the previous step's, whose D_{t-1} the window rule reads). */
 int dkv_step(dkv_cache* cache, const int32_t* tokens, const uint8_t* masked, const int32_t* next_pos, int k,
              int cand_lo, int cand_hi, int rows_bound, float* conf, int32_t* pred, float* logits_dbg,
              void* stream);
@@ -234,7 +241,10 @@ int dkv_select_unmask(const float* conf, const int32_t* pred, int batch, int seq
 int dkv_step_host(dkv_cache* cache, int32_t* tokens_host, uint8_t* masked_host, const int32_t* next_pos_host,
                   int k, int cand_lo, int cand_hi, int rows_bound, int32_t* chosen_host, void* stream);
 
-/* A whole generation on the device with no host synchronisation: T = gen_len/k
+/* The sampling loop of Sec. 3.1 (predict every masked position, keep the most
+ * confident, leave the rest masked) with the semi-autoregressive blocks of the
+ * paper's generation settings (appendix table of L, T and block size), as a
+ * whole generation on the device with no host synchronisation: T = gen_len/k
  * steps of dkv_step + dkv_select_unmask over `tokens` / `masked` (device,
  * updated in place), semi-autoregressive blocks of block_len positions
  * (block_len = 0: one block).  order_dev [T, batch, k] int32 is required for
@@ -247,9 +257,15 @@ int dkv_generate(dkv_cache* cache, int32_t* tokens, uint8_t* masked, const int32
 /* Bookkeeping.  dkv_get_stats synchronises the stream of the last step. */
 int dkv_get_stats(const dkv_cache* cache, dkv_stats* out);
 /* Step number at which each slot was last written (0 = never): device
- * int32 [batch, seq_len]; the one-step delay shows as unmask step + 1. */
+ * int32 [batch, seq_len].  Appendix A: the tokens that newly enter the cache at
+ * step t are those decoded at step t-1, so under Eq. 4 a decoded position shows
+ * its unmask step + 1 until the next refresh (with delay = 0, Eq. 3: its
+ * unmask step); prompt positions under PREFILL / PD show 1. */
 int dkv_get_provenance(const dkv_cache* cache, int32_t* written_step, void* stream);
-/* The index maps of the last step: act_idx [batch*seq_len] (flattened
+/* The token-level index maps of the last step (Appendix A: the reordering is
+ * done once per model evaluation on [B, L] indices and shared by all layers;
+ * Algorithm 1's x' = x[M_{t-1}] and the scatter of the outputs back to their
+ * original positions): act_idx [batch*seq_len] (flattened
  * b*seq_len+pos, ascending; entries past the count are undefined), row_off
  * [batch+1] and inv [batch, seq_len] (compact row of a position, -1 if
  * inactive).  Any pointer may be NULL. */
@@ -257,8 +273,9 @@ int dkv_get_index_maps(const dkv_cache* cache, int32_t* act_idx, int32_t* row_of
 /* Synchronises the stream of the last call and returns DKV_OK, or
  * DKV_E_DEVICE if a kernel set the status word (the word is in *word). */
 int dkv_status(dkv_cache* cache, int32_t* word);
-/* Direct read access to a layer's slots for tests: device pointers to
- * K and V of layer `layer`, layout [batch][kv_head][pos][head_dim]. */
+/* Direct read access to a layer's slots (Algorithm 1's cached Key and Value
+ * states, after RoPE): device pointers to K and V of layer `layer`, layout
+ * [batch][kv_head][pos][head_dim] in the activation type. */
 int dkv_cache_slots(const dkv_cache* cache, int layer, void** k_slots, void** v_slots);
 
 /* Per-kernel-class timing: when enabled, every launch is bracketed by CUDA
@@ -312,12 +329,12 @@ int dkv_op_attention(const void* q, const void* k_slots, const void* v_slots, vo
 /* The same projection GEMM as dkv_op_gemm for callers that cannot allocate
  * device memory.  (The paper has no counterpart: this entry point exists for
  * integration only.)  Some hosts of this library may not call cudaMalloc or
- * any allocator at the point where they need a projection: code running while
- * a stream is being captured into a CUDA graph, a callback on a latency-
- * critical serving thread whose memory pool is fixed at start-up, or a process
- * whose device memory is fully handed to another framework.  For them the
- * split-K partial sums, which dkv_op_gemm keeps in a caller-provided
- * workspace, live in an array compiled into the library image:
+ * any allocator at the point where they need a projection: a callback on a
+ * latency-critical serving thread whose memory pool is fixed at start-up, a
+ * plug-in inside a process whose device memory is fully handed to another
+ * framework, code that runs after the process has been told to stop
+ * allocating.  For them the split-K partial sums, which dkv_op_gemm keeps in a
+ * caller-provided workspace, live in an array compiled into the library image:
  * DKV_STATIC_SCRATCH_BYTES (16 MiB) of device memory on every GPU that loads
  * the library, held until the process exits.
  *   x [rows, K], w [N, K] of the 16-bit `dtype` (DKV_F16 or DKV_BF16), out
@@ -327,13 +344,14 @@ int dkv_op_attention(const void* q, const void* k_slots, const void* v_slots, vo
  * must `splits` slabs when splits is given; otherwise DKV_E_NOMEM and nothing
  * is launched.  With splits = 0 the library picks a count that fits.
  * The first call on each device looks up the array's device address (no
- * allocation; make that first call outside any stream capture).  The function
- * calls no allocator.
+ * allocation) and keeps it in a per-device table indexed by the device
+ * ordinal of the current (primary) context; make that first call before any
+ * stream capture, and not from two host threads at once (the table is filled
+ * without a lock).  The function calls no allocator.
  * Every call on a device uses the SAME array and leaves its partial sums
  * there.  Nothing has to be cleared between calls: each call writes every
  * element it later reads.  Two calls whose kernels can overlap on the GPU
- * (different streams, or graphs replayed concurrently) race on the array and
- * give wrong results: serialise them.
+ * (different streams) race on the array and give wrong results: serialise them.
  * Errors: INVALID_ARG (NULL), UNSUPPORTED (dtype), SHAPE, NOMEM, CUDA. */
 #define DKV_STATIC_SCRATCH_BYTES (16u << 20)
 size_t dkv_static_scratch_bytes(void);

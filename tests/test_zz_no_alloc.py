@@ -2,8 +2,8 @@
 regular one (dkv_op_gemm), through the C ABI.
 
 Who needs it: code that must issue a projection at a moment when it may not
-allocate device memory (during a stream capture, on a serving thread whose
-pool is fixed, inside a process whose memory belongs to another framework).
+allocate device memory (on a serving thread whose pool is fixed at start-up,
+inside a process whose device memory belongs to another framework).
 The entry point keeps the split-K partial sums in a fixed array inside the
 library, so successive calls share that array and see each other's leftovers.
 The test therefore makes two calls in a row with different shapes and checks
