@@ -991,7 +991,11 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       if (rc) return rc;
     }
     Launch lk(c, st, PC_HEAD_STATS, 24.0 * H * ((md.vocab + 31) / 32), 0);
-    launch_k(k_head_combine, H, 256, 0, st, static_cast<const float*>(a.st_max), static_cast<const float*>(a.st_sum),
+    static PerDeviceOnce comb_once;
+    if (comb_once.need() &&
+        cudaFuncSetAttribute(k_head_combine, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess)
+      return DKV_E_CUDA;
+    launch_k(k_head_combine, H, 256, 100 * 1024, st, static_cast<const float*>(a.st_max), static_cast<const float*>(a.st_sum),
              static_cast<const int*>(a.st_arg), static_cast<const float*>(a.st_m2), static_cast<const float*>(a.st_t),
              score, (md.vocab + 31) / 32, H, h_dev, a.head_pos, conf, pred);
     return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;

@@ -489,88 +489,98 @@ k_head_stats(const float* __restrict__ logits, const int* __restrict__ n_head_de
   }
 }
 
-// Combine the per-32-id statistics of the head GEMM: per head row the global
-// max (lowest id on ties), S = sum exp(l - max), and for the margin / entropy
-// scores the second largest logit and T = sum exp(l - max)(l - max); the score
-// is written at the row's original position.  One CTA of 256 threads per row.
+// Softmax statistics of a set of token ids: the largest logit m (its id: lowest on ties), the second
+// largest m2 (over the other ids), S = sum exp(l - m) and T = sum exp(l - m)(l - m).  merge() joins the
+// statistics of two disjoint sets; it is exact in (m, arg, m2) and order-independent there.
+struct HeadStat {
+  float m, m2, s, t;
+  int arg;
+};
+__device__ __forceinline__ HeadStat head_stat_empty() {
+  HeadStat e;
+  e.m = -CUDART_INF_F;
+  e.m2 = -CUDART_INF_F;
+  e.s = 0.f;
+  e.t = 0.f;
+  e.arg = 0x7fffffff;
+  return e;
+}
+__device__ __forceinline__ HeadStat head_stat_merge(const HeadStat& a, const HeadStat& b) {
+  const bool b_wins = b.m > a.m || (b.m == a.m && b.arg < a.arg);
+  const HeadStat& hi = b_wins ? b : a;
+  const HeadStat& lo = b_wins ? a : b;
+  HeadStat r;
+  r.m = hi.m;
+  r.arg = hi.arg;
+  r.m2 = fmaxf(fmaxf(hi.m2, lo.m2), lo.m);
+  if (lo.m == -CUDART_INF_F) {          // an empty side (also when both are empty): nothing to rescale
+    r.s = hi.s;
+    r.t = hi.t;
+  } else {
+    const float dm = lo.m - hi.m;        // <= 0
+    const float w = expf(dm);
+    r.s = hi.s + w * lo.s;
+    r.t = hi.t + w * (lo.t + lo.s * dm);
+  }
+  return r;
+}
+__device__ __forceinline__ HeadStat head_stat_shfl_xor(const HeadStat& v, int o) {
+  HeadStat r;
+  r.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+  r.m2 = __shfl_xor_sync(0xffffffffu, v.m2, o);
+  r.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+  r.t = __shfl_xor_sync(0xffffffffu, v.t, o);
+  r.arg = __shfl_xor_sync(0xffffffffu, v.arg, o);
+  return r;
+}
+
+// Combine the per-32-id statistics of the head GEMM (arrays [ceil(V/32)][ld], one column per head row):
+// one pass per head row with an online merge per thread, then a merge across the block; the score is
+// written at the row's original position.  One CTA of 256 threads per row.  The launch asks for enough
+// dynamic shared memory that an SM holds one block: launched early behind the head GEMM, the blocks would
+// otherwise pile up on the few SMs with room and run several times longer.
 __global__ void __launch_bounds__(256)
 k_head_combine(const float* __restrict__ st_max, const float* __restrict__ st_sum, const int* __restrict__ st_arg,
                const float* __restrict__ st_m2, const float* __restrict__ st_t, int score, int n_groups, int ld,
                const int* __restrict__ n_head_dev, const int32_t* __restrict__ head_pos, float* __restrict__ conf,
                int32_t* __restrict__ pred) {
-  __shared__ float s_m[8];
-  __shared__ int s_i[8];
-  __shared__ float s_s[8], s_t[8], s_m2[8];
+  __shared__ HeadStat s_w[8];
   pdl_enter(15);
   const int i = blockIdx.x;
   if (i >= *n_head_dev) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  float m = -CUDART_INF_F;
-  int mi = 0x7fffffff;
-  for (int g = tid; g < n_groups; g += 256) {
-    const float v = st_max[static_cast<long long>(g) * ld + i];
-    const int a = st_arg[static_cast<long long>(g) * ld + i];
-    if (v > m || (v == m && a < mi)) {
-      m = v;
-      mi = a;
-    }
-  }
-  for (int o = 16; o > 0; o >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, m, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, mi, o);
-    if (om > m || (om == m && oi < mi)) {
-      m = om;
-      mi = oi;
-    }
-  }
-  if (lane == 0) {
-    s_m[warp] = m;
-    s_i[warp] = mi;
-  }
-  __syncthreads();
-  m = s_m[0];
-  mi = s_i[0];
-  for (int w = 1; w < 8; ++w) {
-    if (s_m[w] > m || (s_m[w] == m && s_i[w] < mi)) {
-      m = s_m[w];
-      mi = s_i[w];
-    }
-  }
-  float s = 0.f, t = 0.f, m2 = -CUDART_INF_F;
-  for (int g = tid; g < n_groups; g += 256) {
-    const long long at = static_cast<long long>(g) * ld + i;
-    const float gm = st_max[at];
-    if (gm > -CUDART_INF_F) {
-      const float w = expf(gm - m), gs = st_sum[at];
-      s += gs * w;
-      if (score != SCORE_MAXPROB) {
-        t += w * (st_t[at] + gs * (gm - m));
-        // second largest overall: the group's own second, or its largest if the winner lives elsewhere
-        m2 = fmaxf(m2, st_arg[at] == mi ? st_m2[at] : gm);
+  HeadStat acc = head_stat_empty();
+  for (int g0 = tid; g0 < n_groups; g0 += 4 * 256) {
+    // four groups' loads in flight before any is merged
+    HeadStat v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int g = g0 + u * 256;
+      v[u] = head_stat_empty();
+      if (g < n_groups) {
+        const long long at = static_cast<long long>(g) * ld + i;
+        v[u].m = __ldcg(st_max + at);
+        v[u].arg = __ldcg(st_arg + at);
+        v[u].s = __ldcg(st_sum + at);
+        if (score != SCORE_MAXPROB) {
+          v[u].m2 = __ldcg(st_m2 + at);
+          v[u].t = __ldcg(st_t + at);
+        }
       }
     }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc = head_stat_merge(acc, v[u]);
   }
-  for (int o = 16; o > 0; o >>= 1) {
-    s += __shfl_xor_sync(0xffffffffu, s, o);
-    t += __shfl_xor_sync(0xffffffffu, t, o);
-    m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, o));
-  }
-  if (lane == 0) {
-    s_s[warp] = s;
-    s_t[warp] = t;
-    s_m2[warp] = m2;
-  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc = head_stat_merge(acc, head_stat_shfl_xor(acc, o));
+  if (lane == 0) s_w[warp] = acc;
   __syncthreads();
   if (tid == 0) {
-    float S = 0.f, T = 0.f, M2 = -CUDART_INF_F;
-    for (int w = 0; w < 8; ++w) {
-      S += s_s[w];
-      T += s_t[w];
-      M2 = fmaxf(M2, s_m2[w]);
-    }
+    HeadStat r = s_w[0];
+    for (int w = 1; w < 8; ++w) r = head_stat_merge(r, s_w[w]);
     const int flat = head_pos[i];
-    conf[flat] = head_score(score, m, M2, S, T);
-    pred[flat] = mi;
+    conf[flat] = head_score(score, r.m, r.m2, r.s, r.t);
+    pred[flat] = r.arg;
   }
 }
 
