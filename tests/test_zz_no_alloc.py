@@ -34,13 +34,15 @@ def test_static_scratch_gemm_matches_workspace_gemm_on_two_calls_in_a_row():
         x, w = case(rows, n, k, dtype, seed)
         ref = torch.empty(rows, n, dtype=torch.float32, device="cuda")
         got = torch.full((rows, n), float("nan"), dtype=torch.float32, device="cuda")
-        B.dkv_op_gemm(x, w, ref, dtype, splits)
+        workspace = B.dkv_op_gemm(x, w, ref, dtype, splits)
         torch.cuda.synchronize()
-        # the entry point must not allocate: neither through torch's allocator nor from the device
+        # the entry point must not allocate: torch's allocator must not grow and the device's free memory
+        # must not shrink across the call (every tensor of the test is alive on both sides of it)
         held, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         B.dkv_op_gemm_static(x, w, got, dtype, splits)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == held and torch.cuda.mem_get_info()[0] == free_before
+        assert torch.cuda.memory_allocated() <= held and torch.cuda.mem_get_info()[0] >= free_before
+        del workspace
         exact = x.float().cpu().numpy().astype(np.float64) @ w.float().cpu().numpy().astype(np.float64).T
         # same tolerance as the GEMM parity tests: fp32 accumulation order only
         np.testing.assert_allclose(got.cpu().numpy(), ref.cpu().numpy(), atol=3e-6 * k ** 0.5 * 4, rtol=1e-5)
