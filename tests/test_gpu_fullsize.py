@@ -65,6 +65,38 @@ def test_llada_shaped_two_layers_isolated_prefill_pd():
     print("llada 2-layer isolated prefill worst err/sigma", worst)
 
 
+def test_llada_shaped_two_layers_greedy_long_sequence():
+    """Config 4's shape at depth 2: prompt 128 + 1024 masked (L = 1152, nine 128-slot tiles), Greedy with a
+    window of 4 and a refresh every 2 steps over a seeded order: a full step over 1152 rows (five row
+    tiles, multi-wave launches: the row kernels), then steps of at most 6 rows (one-wave launches: the
+    fused tails), one head row per step."""
+    ms, P, G = synth.llada_shape(2), 128, 1024
+    pol = O.Policy(O.POLICY_GREEDY, 2, window=4)
+    W, model = U.build_pair(ms, 5, True, oracle_dtype=np.float32)
+    prompt = synth.make_prompt(1, P, ms.vocab - 1, 5)
+    order = synth.random_order(1, P, G, 1, 5)
+    sampler = O.Sampler(U.oracle_model(ms), W, prompt[0], G, 1, pol, None, order[:, 0, :], form="slots",
+                        keep_logits=True, dtype=np.float32)
+    run = U.ForcedRun(ms, model, 1, P, G, pol, 1, fused=True)
+    worst = 0.0
+    for _ in range(4):
+        st = sampler.step()
+        assert st.t == 1 or st.t % 2 == 1 or len(st.active) <= 6
+        err, sig, conf, pred = U.compare_step(run, [st], True, logit_tol_sigma=BF16_TOL_SIGMA)
+        worst = max(worst, err / sig)
+    assert B.dkv_status(run.cache) == 0 and B.dkv_status(run.cache_f) == 0
+    print("llada 2-layer greedy L=1152 worst err/sigma", worst)
+
+
+def test_dream_shaped_full_depth_parity_first_steps():
+    """All 28 Dream-7B-shaped layers (GQA 28 query / 4 KV heads, FFN 18944, vocabulary 152064), PD with two
+    tokens per step: the joint full step, a cached step and the generation-only refresh, logits within
+    2e-2 sigma, both head paths, identical index maps."""
+    worst = forced(synth.dream_shape(28), 1, 96, 64, 2, O.Policy(O.POLICY_PD, 2), None, 3, seed=2)
+    print("dream 28-layer worst err/sigma", worst)
+    assert worst < BF16_TOL_SIGMA
+
+
 def test_llada_shaped_interval_one_equals_no_cache_on_device():
     ms = synth.llada_shape(1)
     w = synth.make_weights(ms, 2, "bfloat16", "cuda")
