@@ -303,6 +303,19 @@ int dkv_profile_read(dkv_cache* cache, dkv_profile_entry* out, int* n);
  * records = NULL switches the trace off.  Synchronises the device. */
 int dkv_trace_set(void* records, int capacity);
 
+/* Test hook for the error path of the bounded waits (failure detection
+ * without a GPU fault): in a fused projection launch the thread blocks of a
+ * weight tile wait for each other, at most `wait_cycles` SM clocks (default:
+ * about two seconds).  With never_complete != 0 they expect one arrival more
+ * than will ever come, so that every such wait runs out after wait_cycles:
+ * the kernels skip the row work that depended on it, finish normally and set
+ * bit 3 (value 8) of the status word; the step's results are then meaningless
+ * and the arrival counters are left non-zero, so the handle must be destroyed
+ * and a new one initialised (dkv_init_cache clears them) before the arena is
+ * used again.  Nothing traps and no kernel is left waiting.  Errors:
+ * INVALID_ARG (wait_cycles outside [1000, default]), STATE. */
+int dkv_debug_tail_wait(dkv_cache* cache, long long wait_cycles, int never_complete);
+
 /* ---- kernel-level entry points (single-layer sweeps and unit parity) ---- */
 
 /* out[r, n] = sum_k x[r, k] * w[n, k] for r < rows: the projection GEMM used

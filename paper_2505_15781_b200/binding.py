@@ -29,7 +29,7 @@ EXPORTS = [
     "dkv_cache_destroy", "dkv_step", "dkv_refresh", "dkv_select_unmask", "dkv_step_host", "dkv_generate",
     "dkv_get_stats", "dkv_get_provenance", "dkv_get_index_maps", "dkv_status", "dkv_cache_slots",
     "dkv_profile_enable", "dkv_profile_read", "dkv_gemm_workspace_bytes", "dkv_op_gemm", "dkv_op_attention",
-    "dkv_static_scratch_bytes", "dkv_op_gemm_static", "dkv_trace_set",
+    "dkv_static_scratch_bytes", "dkv_op_gemm_static", "dkv_trace_set", "dkv_debug_tail_wait",
 ]
 
 
@@ -112,6 +112,7 @@ def load():
     lib.dkv_op_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.dkv_op_attention.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
     lib.dkv_trace_set.argtypes = [vp, i32]
+    lib.dkv_debug_tail_wait.argtypes = [vp, C.c_longlong, i32]
     lib.dkv_static_scratch_bytes.restype = sz
     lib.dkv_static_scratch_bytes.argtypes = []
     lib.dkv_op_gemm_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
@@ -347,6 +348,10 @@ def dkv_op_gemm_static(x, w, out, dtype: int, splits: int = 0, stream=None):
     n = w.shape[0]
     _check("dkv_op_gemm_static", load().dkv_op_gemm_static(_ptr(x), _ptr(w), _ptr(out), rows, n, k, dtype, splits,
                                                            _stream(stream)))
+
+
+def dkv_debug_tail_wait(cache: Cache, wait_cycles: int, never_complete: bool):
+    _check("dkv_debug_tail_wait", load().dkv_debug_tail_wait(cache.handle, wait_cycles, 1 if never_complete else 0))
 
 
 def dkv_trace_set(records, capacity: int):

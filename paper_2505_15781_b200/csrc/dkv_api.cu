@@ -369,6 +369,8 @@ struct dkv_cache {
   bool attn_tc;
   int fuse_tails;        // bit 0: RoPE / K/V scatter inside the QKV GEMM; bit 1: residual / norm statistics inside
                          // the O and down GEMMs (one-wave launches)
+  long long tail_wait_cycles;   // bound of the fused tails' cross-CTA wait; dkv_debug_tail_wait shortens it
+  int tail_extra;               // arrivals the tails expect beyond the real ones (0; 1 under dkv_debug_tail_wait)
   int step;              // steps run so far
   int last_refresh;      // step number of the last full / generation-only step
   int pending_refresh;   // -1 none, else DKV_REFRESH_*
@@ -558,6 +560,8 @@ struct RowScale {
 struct FusedTail {
   int mode = FUSE_NONE;
   unsigned int* tile_cnt = nullptr;
+  long long wait_cycles = GEMM_WAIT_CYCLES;
+  int extra = 0;
   float* h = nullptr;
   const float* gain = nullptr;
   void* xn_out = nullptr;
@@ -684,6 +688,8 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
     const FusedTail& t = o.tail;
     p.fuse_mode = t.mode;
     p.tile_cnt = t.tile_cnt;
+    p.tail_wait_cycles = t.wait_cycles;
+    p.tail_extra = t.extra;
     p.h = t.h;
     p.gain = t.gain;
     p.xn_out = t.xn_out;
@@ -827,6 +833,8 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     if (c->fuse_tails & 2) {
       o.tail.mode = FUSE_RESID;
       o.tail.tile_cnt = a.tile_cnt;
+      o.tail.wait_cycles = c->tail_wait_cycles;
+      o.tail.extra = c->tail_extra;
       o.tail.h = a.h;
       o.tail.gain = gain;
       o.tail.xn_out = a.xn;
@@ -862,6 +870,8 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     if ((c->fuse_tails & 1) && R <= 256) {
       o.tail.mode = FUSE_QKV;
       o.tail.tile_cnt = a.tile_cnt;
+      o.tail.wait_cycles = c->tail_wait_cycles;
+      o.tail.extra = c->tail_extra;
       o.tail.act_idx = a.act_idx;
       o.tail.rope_tab = a.rope_tab;
       o.tail.seq_len = dm.L;
@@ -1361,6 +1371,8 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   }
   // read per handle (not once per process), so that a test can build handles of both kinds
   c->fuse_tails = env_int("DKV_FUSE_TAILS", 3);
+  c->tail_wait_cycles = GEMM_WAIT_CYCLES;
+  c->tail_extra = 0;
   c->step = 0;
   c->last_refresh = 1;
   c->pending_refresh = -1;
@@ -1547,6 +1559,14 @@ int dkv_profile_read(dkv_cache* c, dkv_profile_entry* out, int* n) {
     c->prof[i].launches = 0;
     c->prof[i].ms = c->prof[i].bytes = c->prof[i].flops = 0.0;
   }
+  return DKV_OK;
+}
+
+int dkv_debug_tail_wait(dkv_cache* c, long long wait_cycles, int never_complete) {
+  DKV_CHECK_CACHE(c);
+  if (wait_cycles < 1000 || wait_cycles > GEMM_WAIT_CYCLES) return DKV_E_INVALID_ARG;
+  c->tail_wait_cycles = wait_cycles;
+  c->tail_extra = never_complete ? 1 : 0;
   return DKV_OK;
 }
 

@@ -132,6 +132,9 @@ struct GemmTcParams {
   // fused row epilogue across the CTAs of a weight tile (FUSE_*); needs units <= resident CTAs
   int fuse_mode;
   unsigned int* tile_cnt;  // [weight tiles * row tiles] arrival counters, zero between launches
+  long long tail_wait_cycles;  // bound of the wait for the tile's other CTAs (GEMM_WAIT_CYCLES unless a test shortens it)
+  int tail_extra;          // arrivals expected beyond the tile's K splits: 0; a test of the error path sets 1,
+                           // so that the wait can only run out
   // FUSE_RESID
   float* h;                // [rows][n] residual stream, updated in place
   const float* gain;       // [n] gains of the norm that follows
@@ -628,8 +631,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         if (et == 0) {
           atomicAdd(cnt, 1u);
           const long long t0 = clock64();
-          while (ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits)) {
-            if (*abort_flag || clock64() - t0 > GEMM_WAIT_CYCLES) {
+          while (ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits + p.tail_extra)) {
+            if (*abort_flag || clock64() - t0 > p.tail_wait_cycles) {
               fail = true;
               *abort_flag = 1;
               break;

@@ -219,3 +219,28 @@ def test_greedy_rejects_a_change_of_k_between_steps():
     assert e.value.status == -2
     B.dkv_step(cache, x, m, d, 2, 8, 16, 8, conf, pred)
     assert B.dkv_status(cache) == 0
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """The bounded waits' error path, without a fault: the fused tails of one handle are told to expect an
+    arrival that never comes and to give up after 2 million clocks (about a millisecond).  The step must
+    come back, dkv_status must show the wait bit (8), and a fresh handle on the same device must then
+    reproduce the oracle."""
+    ms, P, G, pol = HD128, 20, 12, O.Policy(O.POLICY_DECODE, 0)
+    W, model = U.build_pair(ms, 6, True)
+    x, m = synth.initial_state(synth.make_prompt(1, P, ms.vocab - 1, 6), G, ms.mask_id)
+    tx, tm = torch.from_numpy(x).cuda(), torch.from_numpy(m).cuda()
+    conf = torch.empty(1, P + G, device="cuda")
+    pred = torch.empty(1, P + G, dtype=torch.int32, device="cuda")
+    cache = B.dkv_init_cache(model, 1, P + G, P, U.gpu_policy(pol))
+    B.dkv_debug_tail_wait(cache, 2_000_000, True)
+    B.dkv_step(cache, tx, tm, None, 1, P, P + G, G, conf, pred)
+    torch.cuda.synchronize()
+    assert B.dkv_status(cache) & 8
+    del cache
+    prompt = synth.make_prompt(1, P, ms.vocab - 1, 6)
+    sampler = O.Sampler(U.oracle_model(ms), W, prompt[0], G, 1, pol, None, None, "literal", keep_logits=True)
+    run = U.ForcedRun(ms, model, 1, P, G, pol, 1, fused=True)
+    for _ in range(2):
+        U.compare_step(run, [sampler.step()], False, logit_tol_sigma=2e-2)
+    assert B.dkv_status(run.cache) == 0 and B.dkv_status(run.cache_f) == 0
