@@ -5,10 +5,10 @@
 // memory).  Per 32 KB of weights a CTA therefore holds br * 64 bytes of rows
 // instead of br * 128: the ring is deeper at the same shared memory and the
 // L2 -> SM traffic of the rows halves, which is what bounds the one-CTA kernel
-// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).  Which 128 rows a CTA
-// stages for MMA h is a matter of its TMA coordinate only: plain launches take rows
-// [h*256 + rank*128, +128) so that the tile is covered in order; the SwiGLU launch takes rows
-// [rank*256 + h*128, +128) of a weight copy grouped [128 gate | 128 up] per 256 rows, so that each CTA
+// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).  The kernel serves ONE
+// launch: the unsplit gate/up projection with the SwiGLU epilogue (the split-K launches gain nothing from
+// pairs).  Which 128 rows a CTA stages for MMA h is a matter of its TMA coordinate only: rank r takes rows
+// [r*256 + h*128, +128) of the weight copy grouped [128 gate | 128 up] per 256 rows, so that each CTA
 // holds the gate rows (MMA 0) and the up rows (MMA 1) of the same 128 features.
 //
 // Roles per CTA (320 threads): warp 0 = TMA producer of its own half of the
@@ -177,8 +177,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         const uint32_t a_dst = smem_base + s * p.stage_bytes;
         for (int h = 0; h < 2; ++h)
           tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, (c.kb0 + c.i) * GEMM_BK,
-                                c.n0 + (p.swiglu_out ? static_cast<int>(rank) * 256 + h * GEMM_BM
-                                                     : h * 256 + static_cast<int>(rank) * GEMM_BM), pol_w);
+                                c.n0 + static_cast<int>(rank) * 256 + h * GEMM_BM, pol_w);
       };
       auto load_b = [&](const Cursor& c, int it) {
         const int s = it % STAGES;
@@ -285,10 +284,9 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
       ok = mbar_wait_bounded(smem_u32(&acc_full[buf]), use & 1, abort_flag, GEMM_WAIT_CYCLES);
       if (!ok) break;
       tc_fence_after();
-      float* out = p.out + static_cast<long long>(split) * p.split_stride;
-      const int row_in_tile = static_cast<int>(rank) * GEMM_BM + q * 32 + lane;   // + h * 256
+      const int row_in_tile = static_cast<int>(rank) * GEMM_BM + q * 32 + lane;
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(buf * 2 * p.col_stride);
-      if (p.swiglu_out) {
+      {
         // the gate/up copy is grouped [128 gate rows | 128 up rows] per 256 rows and this CTA staged the
         // gate rows (MMA 0) and the up rows (MMA 1) of features (n0 / 2) + rank * 128 + [0, 128)
         const int jf = (n0 >> 1) + row_in_tile;
@@ -326,78 +324,6 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
 #pragma unroll
               for (int jj = 0; jj < 16; ++jj)
                 if (jj < n_ok) dst[static_cast<long long>(jj) * p.ld_u] = bits[jj];
-            }
-          }
-        }
-      } else
-      for (int h = 0; h < 2; ++h) {
-        const int n = n0 + h * 256 + row_in_tile;
-        const uint32_t t_addr = t_lane + static_cast<uint32_t>(h * p.col_stride);
-        for (int c = cs * 16; c < p.br; c += 32) {
-          if (r0 + c >= r_valid) break;
-          uint32_t v[16];
-          if (n_kb > 0) {
-            tmem_ld_x16(t_addr + c, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) v[jj] = __float_as_uint(__uint_as_float(v[jj]) * s_rs[c + jj]);
-          } else {
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) v[jj] = 0u;
-          }
-          if (p.head_mode) {
-            // softmax statistics over this warp's 32 token ids, per row, by warp shuffles
-            const bool live = n < p.n && n != p.mask_id;
-            const long long slot = static_cast<long long>((n0 + h * 256 + static_cast<int>(rank) * GEMM_BM) / 32 + q) * p.r_bound;
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-              const float val = live ? __uint_as_float(v[jj]) : -INFINITY;
-              float m = val;
-              int arg = live ? n : 0x7fffffff;
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) {
-                const float om = __shfl_xor_sync(0xffffffffu, m, o);
-                const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
-                if (om > m || (om == m && oa < arg)) {
-                  m = om;
-                  arg = oa;
-                }
-              }
-              float e = live ? expf(val - m) : 0.f;
-              float m2 = -INFINITY, tt = 0.f;
-              if (p.st_m2) {
-                m2 = (live && n != arg) ? val : -INFINITY;
-                tt = live ? e * (val - m) : 0.f;
-              }
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-              if (p.st_m2) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                  m2 = fmaxf(m2, __shfl_xor_sync(0xffffffffu, m2, o));
-                  tt += __shfl_xor_sync(0xffffffffu, tt, o);
-                }
-              }
-              const int r = r0 + c + jj;
-              if (lane == jj && r < r_valid) {
-                p.st_max[slot + r] = m;
-                p.st_sum[slot + r] = e;
-                p.st_arg[slot + r] = arg;
-                if (p.st_m2) {
-                  p.st_m2[slot + r] = m2;
-                  p.st_t[slot + r] = tt;
-                }
-              }
-            }
-          } else if (n < p.n) {
-            float* dst = out + static_cast<long long>(r0 + c) * p.ldo + n;
-            if (r0 + c + 16 <= r_valid) {
-#pragma unroll
-              for (int jj = 0; jj < 16; ++jj) dst[static_cast<long long>(jj) * p.ldo] = __uint_as_float(v[jj]);
-            } else {
-#pragma unroll
-              for (int jj = 0; jj < 16; ++jj)
-                if (r0 + c + jj < r_valid) dst[static_cast<long long>(jj) * p.ldo] = __uint_as_float(v[jj]);
             }
           }
         }
