@@ -126,10 +126,6 @@ int make_tmap_nd(CUtensorMap* tm, const void* base, int rank, const cuuint64_t* 
   return r == CUDA_SUCCESS ? DKV_OK : DKV_E_CUDA;
 }
 
-// Tensor maps of the tcgen05 attention kernel (head_dim 128): queries [rows][H_q][128] with a box of
-// (64 columns, the KV head's query heads, rows_q rows); K and V slots as [all rows][128].
-int env_int(const char* name, int dflt);
-
 // The opt-in to large dynamic shared memory is a per-device property of a kernel: one flag per
 // (call site, device), so that a process that drives several GPUs sets it on each of them.
 struct PerDeviceOnce {
@@ -148,6 +144,8 @@ struct AttnMaps {
   CUtensorMap k64, v64;     // K/V boxes of 64 slots (two CTAs per SM)
   int group, rows_q;
 };
+// Tensor maps of the tcgen05 attention kernel (head_dim 128): queries [rows][H_q][128] with a box of
+// (64 columns, the KV head's query heads, rows_q rows);
 // K and V slots as a 3-D tensor [KV heads of all layers and sequences][kv_len slots][128]: a slot tile that
 // reaches past kv_len is zero-filled by the copy engine instead of running into the next head's (or the
 // next layer's, possibly unwritten) slots.  kv_stride = slots per head in memory (>= kv_len).
