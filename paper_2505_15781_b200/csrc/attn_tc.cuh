@@ -32,12 +32,19 @@ constexpr int ATC_BKV = 128;      // slots per iteration of the one-CTA-per-SM s
 constexpr int ATC_DH = 128;
 constexpr int ATC_THREADS = 320;     // TMA warp, MMA warp, two softmax warpgroups (the larger shape)
 constexpr int ATC_TILE = 128 * 128;                 // bytes of a [128 rows x 64 columns] 16-bit tile
-// Q (2 tiles) | K,V: 2 stages x (2 + 2) half tiles of [BKV slots x 64 columns] | P (NWG tiles) |
-// barriers | row maxima / sums exchanged by two warpgroups.  The two-CTA shape has no room for
-// alignment slack: its dynamic shared memory must start on a 1024-byte boundary (checked).
+// Q (2 tiles) | K,V: 2 stages x (2 + 2) half tiles of [BKV slots x 64 columns] | P (NPB buffers of NWG
+// tiles) | barriers | row maxima / sums exchanged by two warpgroups.  There is no room for alignment
+// slack: the dynamic shared memory must start on a 1024-byte boundary (checked).
+// The one-CTA-per-SM shape keeps TWO P buffers: its launches are chains of dependent iterations, and
+// with one buffer the softmax of tile j+1 could not publish its P before P_j V_j had completed.
+template <int NWG>
+__host__ __device__ constexpr int attn_tc_pbufs() {
+  return NWG == 2 ? 2 : 1;
+}
 template <int BKV, int NWG>
 constexpr int attn_tc_smem() {
-  return 2 * ATC_TILE + 2 * 4 * BKV * 128 + NWG * ATC_TILE + 256 + (NWG == 2 ? 1024 + 2 * 2 * 128 * 4 : 0);
+  return 2 * ATC_TILE + 2 * 4 * BKV * 128 + attn_tc_pbufs<NWG>() * NWG * ATC_TILE + 256 +
+         (NWG == 2 ? 2 * 2 * 128 * 4 : 0);
 }
 constexpr int ATC_SMEM = attn_tc_smem<128, 2>();
 constexpr long long ATC_WAIT_CYCLES = 4000000000LL;
@@ -114,13 +121,14 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   static_assert(BKV == 64 * NWG, "each softmax thread owns 64 slots of a tile");
   constexpr int KVT = BKV * 128;                        // bytes of a [BKV slots x 64 columns] half tile
   constexpr int TMEM_COLS = (2 * BKV + ATC_DH) > 256 ? 512 : 256;
+  constexpr int NPB = attn_tc_pbufs<NWG>();             // P buffers
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  const uint32_t smem_base = (NWG == 2) ? ((smem_u32(smem_raw) + 1023u) & ~1023u) : smem_u32(smem_raw);
-  uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t smem_base = smem_u32(smem_raw);
+  uint8_t* smem_al = smem_raw;
   const uint32_t sQ = smem_base;                       // 2 halves (head_dim 0..63, 64..127)
   const uint32_t sKV = sQ + 2 * ATC_TILE;              // stage s: K half0, K half1, V half0, V half1
-  const uint32_t sP = sKV + 8 * KVT;                   // NWG half tiles of 64 slots
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + 2 * ATC_TILE + 8 * KVT + NWG * ATC_TILE);
+  const uint32_t sP = sKV + 8 * KVT;                   // NPB buffers of NWG half tiles of 64 slots
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + 2 * ATC_TILE + 8 * KVT + NPB * NWG * ATC_TILE);
   // K and V tiles have barriers of their own: a K tile is free as soon as its S = Q K^T is done,
   // one iteration before the V tile of the same slots, so the next K load starts that much earlier
   uint64_t* q_full = bars;           // 1
@@ -129,9 +137,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
   uint64_t* v_full = bars + 5;       // 2
   uint64_t* v_empty = bars + 7;      // 2
   uint64_t* s_full = bars + 9;       // 2
-  uint64_t* p_ready = bars + 11;     // 1
-  uint64_t* o_done = bars + 12;      // 1
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  uint64_t* p_ready = bars + 11;     // 2: P buffer b holds the probabilities of its next tile
+  uint64_t* p_free = bars + 13;      // 2: the P V MMAs that read buffer b (and all MMAs before them) are done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 15);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* xch = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);   // NWG == 2: [2][2][128]
 
@@ -146,8 +154,10 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       mbar_init(smem_u32(&v_empty[s]), 1);
       mbar_init(smem_u32(&s_full[s]), 1);
     }
-    mbar_init(smem_u32(p_ready), 4 * NWG);
-    mbar_init(smem_u32(o_done), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&p_ready[b]), 4 * NWG);
+      mbar_init(smem_u32(&p_free[b]), 1);
+    }
     // swizzled tiles need the 1024-byte alignment; without it nothing is loaded and the launch reports
     *abort_flag = (smem_base & 1023u) ? 1 : 0;
     fence_barrier_init();
@@ -229,19 +239,20 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
           tc_fence_after();
           issue_s(j + 1);   // its S buffer was drained before p_ready of iteration j-1
         }
-        ok = mbar_wait_bounded(smem_u32(p_ready), j & 1, abort_flag, ATC_WAIT_CYCLES) &&
+        const int pb = j % NPB;
+        ok = mbar_wait_bounded(smem_u32(&p_ready[pb]), (j / NPB) & 1, abort_flag, ATC_WAIT_CYCLES) &&
              mbar_wait_bounded(smem_u32(&v_full[j & 1]), (j >> 1) & 1, abort_flag, ATC_WAIT_CYCLES);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vbase = sKV + (j & 1) * 4 * KVT + 2 * KVT;
 #pragma unroll
         for (int ks = 0; ks < BKV / 16; ++ks) {   // 16 slots per MMA
-          const uint64_t adesc = umma_desc_sw128(sP + (ks >> 2) * ATC_TILE) + 2 * (ks & 3);
+          const uint64_t adesc = umma_desc_sw128(sP + (pb * NWG + (ks >> 2)) * ATC_TILE) + 2 * (ks & 3);
           const uint64_t bdesc = umma_desc_sw128_mn(vbase + ks * 2048, KVT);
           umma_f16(tO, adesc, bdesc, idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(smem_u32(&v_empty[j & 1]));   // V_j and P_j have been consumed
-        umma_commit(smem_u32(o_done));
+        umma_commit(smem_u32(&p_free[pb]));
       }
     }
   } else if (active) {
@@ -329,13 +340,19 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       }
       const float sum = ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
       l_run = l_run * alpha + sum;
-      if (j > 0) {
-        // P_{j-1} V_{j-1} must be complete before O is rescaled and before P is overwritten
-        ok = mbar_wait_bounded(smem_u32(o_done), (j - 1) & 1, abort_flag, ATC_WAIT_CYCLES);
+      const int pb = j % NPB;
+      if (j >= NPB) {
+        // the P V MMAs that read this P buffer (tile j - NPB) must be complete before it is overwritten
+        ok = mbar_wait_bounded(smem_u32(&p_free[pb]), ((j - NPB) / NPB) & 1, abort_flag, ATC_WAIT_CYCLES);
         if (!ok) continue;        // two warpgroups: reported to everyone at the next iteration's barrier
-        tc_fence_after();
-        // the accumulator only needs touching when some row of this warp moved its exponent
+      }
+      if (j > 0) {
+        // the accumulator only needs touching when some row of this warp moved its exponent; then
+        // P_{j-1} V_{j-1} (and with it every earlier MMA) must be complete first
         if (!__all_sync(0xffffffffu, alpha == 1.f)) {
+          ok = mbar_wait_bounded(smem_u32(&p_free[(j - 1) % NPB]), ((j - 1) / NPB) & 1, abort_flag, ATC_WAIT_CYCLES);
+          if (!ok) continue;
+          tc_fence_after();
 #pragma unroll
           for (int hf = 0; hf < O_COLS / 64; ++hf) {
             uint32_t acc[4][16];
@@ -355,7 +372,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       }
       // P_j -> shared memory, K-major rows of 128 bytes with the 128-byte swizzle; the thread's
       // 64 slots are one 64-column half tile
-      uint8_t* prow = smem_al + (sP - smem_base) + wg * ATC_TILE + (row >> 3) * 1024 + (row & 7) * 128;
+      uint8_t* prow = smem_al + (sP - smem_base) + (pb * NWG + wg) * ATC_TILE + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {            // 16-byte chunks of 8 slots
         const uint32_t* sv = &raw[ch >> 1][(ch & 1) * 8];
@@ -369,12 +386,13 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
       fence_proxy_async_smem();      // the MMA reads P through the async proxy
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(p_ready));
+      if (lane == 0) mbar_arrive(smem_u32(&p_ready[pb]));
     }
     // Leaving the loop with two warpgroups: either every thread finished it or a failed wait was seen
     // by all of them at a barrier; the barrier below is reached by all 256 threads in every case.
     if (n_iter > 0) {
-      ok = ok && mbar_wait_bounded(smem_u32(o_done), (n_iter - 1) & 1, abort_flag, ATC_WAIT_CYCLES);
+      ok = ok && mbar_wait_bounded(smem_u32(&p_free[(n_iter - 1) % NPB]), ((n_iter - 1) / NPB) & 1, abort_flag,
+                                   ATC_WAIT_CYCLES);
       float l_row = l_run;
       if constexpr (NWG == 2) {
         xch[wg * 128 + row] = l_run;
