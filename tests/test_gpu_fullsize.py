@@ -177,6 +177,71 @@ def test_full_depth_properties_in_the_benchmark_configuration():
     torch.cuda.synchronize()
     assert int(pick.item()) == int(chosen[16, 0, 0].item())
     assert int(x1[0, int(pick.item())].item()) == int(xs[int(pick.item())])
+    # a second run of the same 18 steps must reproduce tokens and order bit for bit: the K splits of
+    # the fused launches are summed in a fixed order, whichever CTA arrives first
+    again = B.dkv_init_cache(model, 1, L, P, pol)
+    x2, m2 = torch.from_numpy(x0).cuda(), torch.from_numpy(m0).cuda()
+    chosen2 = torch.full((G, 1, 1), -1, dtype=torch.int32, device="cuda")
+    B.dkv_generate(again, x2, m2, None, 1, 32, steps, chosen2)
+    torch.cuda.synchronize()
+    assert B.dkv_status(again) == 0
+    np.testing.assert_array_equal(x2.cpu().numpy(), x.cpu().numpy())
+    np.testing.assert_array_equal(chosen2.cpu().numpy(), chosen.cpu().numpy())
+
+
+def test_dream_full_size_pd_properties_and_run_to_run_identity():
+    """Config 3 at its full size in the benchmark's launch configuration (28 Dream-shaped layers, batch 4,
+    prompt 512 + 256 masked, two tokens per step, PD with a generation-only refresh every 16 steps).  The
+    oracle cannot run this inside a test, so what holds at any size is checked: the active-row counts of
+    the PD rule, provenance (prompt rows keep step 1's K/V forever; a decoded row is re-stamped one step
+    after it was unmasked; a refresh re-stamps the generation rows only), two distinct candidates chosen
+    per sequence per step, and that a second run of the same generation reproduces the first bit for bit
+    (the cross-CTA reductions of the fused launches have a fixed summation order)."""
+    ms = synth.dream_shape(28)
+    w = synth.make_weights(ms, 0, "bfloat16", "cuda")
+    model = B.dkv_model_create(ms, w, B.DKV_BF16)
+    del w
+    Bn, P, G, k, N, steps = 4, 512, 256, 2, 16, 19
+    L = P + G
+    x0, m0 = synth.initial_state(synth.make_prompt(Bn, P, ms.vocab - 1, 0), G, ms.mask_id)
+    pol = B.make_policy(B.DKV_POLICY_PD, N, max_head_rows=G, max_k=k)
+    runs = []
+    for rep in range(2):
+        cache = B.dkv_init_cache(model, Bn, L, P, pol)
+        x, m = torch.from_numpy(x0).cuda(), torch.from_numpy(m0).cuda()
+        chosen = torch.full((G // k, Bn, k), -1, dtype=torch.int32, device="cuda")
+        prov = torch.empty(Bn, L, dtype=torch.int32, device="cuda")
+        row_off = torch.empty(Bn + 1, dtype=torch.int32, device="cuda")
+        unmask_step = np.zeros((Bn, L), dtype=np.int64)
+        for s_i in range(steps):
+            B.dkv_generate(cache, x, m, None, k, 0, 1, chosen)
+            B.dkv_get_index_maps(cache, None, row_off, None)
+            B.dkv_get_provenance(cache, prov)
+            torch.cuda.synchronize()
+            if rep:
+                continue                      # the second run is only compared with the first
+            t = s_i + 1
+            ro = row_off.cpu().numpy()
+            expect = L if s_i == 0 else (G if s_i % N == 0 else (G - s_i * k) + k)
+            assert (np.diff(ro) == expect).all(), (t, ro)
+            ch = chosen[s_i].cpu().numpy()
+            pv = prov.cpu().numpy()
+            last_refresh = (s_i // N) * N + 1
+            masked = m.cpu().numpy().astype(bool)
+            for b in range(Bn):
+                assert len(set(ch[b])) == k and (ch[b] >= P).all() and (unmask_step[b, ch[b]] == 0).all()
+                unmask_step[b, ch[b]] = t
+                assert (pv[b, :P] == 1).all()                                   # prompt: step 1, never again
+                gen = np.arange(P, L)
+                active_now = masked[b, gen] | np.isin(gen, ch[b])
+                assert (pv[b, gen][active_now] == t).all()
+                stable = gen[~active_now]
+                want = np.where(unmask_step[b, stable] + 1 > last_refresh, unmask_step[b, stable] + 1, last_refresh)
+                np.testing.assert_array_equal(pv[b, stable], want)
+        assert B.dkv_status(cache) == 0
+        runs.append((x.cpu().numpy(), chosen.cpu().numpy()))
+    np.testing.assert_array_equal(runs[0][0], runs[1][0])
+    np.testing.assert_array_equal(runs[0][1], runs[1][1])
 
 
 def test_llada_shaped_full_depth_parity_first_steps():
