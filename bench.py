@@ -327,21 +327,35 @@ def run_ours(args, rank, world):
     pk = peaks()
     roofline, roofline_tensor, roofline_attn, classes = None, None, None, {}
     if rank == 0:
-        job.restart()
-        job.run_steps(first)
-        torch.cuda.synchronize()
-        B.dkv_profile_enable(job.cache, True)
-        agg = {"cached": {}, "refresh": {}}
-
-        def cb(s):
-            bucket = agg["refresh" if job.is_refresh(s) else "cached"]
-            for e in B.dkv_profile_read(job.cache):
-                a = bucket.setdefault(e["name"], dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
-                for key in ("launches", "ms", "bytes", "flops"):
-                    a[key] += e[key]
         n_prof = min(K, job.T)
-        job.run_steps(n_prof, profile_cb=cb)
-        B.dkv_profile_enable(job.cache, False)
+
+        def profile_pass():
+            """Events around every launch of steps first .. first + n_prof - 1, by step kind and kernel class."""
+            job.restart()
+            job.run_steps(first)
+            torch.cuda.synchronize()
+            B.dkv_profile_enable(job.cache, True)
+            res = {"cached": {}, "refresh": {}}
+
+            def cb(s):
+                bucket = res["refresh" if job.is_refresh(s) else "cached"]
+                for e in B.dkv_profile_read(job.cache):
+                    a = bucket.setdefault(e["name"], dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
+                    for key in ("launches", "ms", "bytes", "flops"):
+                        a[key] += e[key]
+            job.run_steps(n_prof, profile_cb=cb)
+            B.dkv_profile_enable(job.cache, False)
+            return res
+        agg = profile_pass()
+        # The same pass with the row tails as kernels of their own (DKV_FUSE_TAILS=0 is read when a handle
+        # is created): the GEMM launches then hold the projection alone, which is what a per-launch
+        # weight-streaming fraction should be read against; the tails show up as row-kernel classes.
+        os.environ["DKV_FUSE_TAILS"] = "0"
+        try:
+            agg_plain = profile_pass()
+        finally:
+            del os.environ["DKV_FUSE_TAILS"]
+            job.restart()
         ms_shape = job.ms
 
         # weight bytes of one launch of each GEMM class (the hot-path table's per-unit figure: 2 K N)
@@ -378,6 +392,19 @@ def run_ours(args, rank, world):
                         "traffic": traffic, "traffic_source": NCU_GEMM_TRAFFIC_SOURCE,
                         "launches": gc["launches"], "avg_launch_us": gc["ms"] * 1e3 / gc["launches"],
                         "algorithmic_bytes_per_launch": gc["weight_bytes"] / gc["launches"]}
+            gp = gemm_sum(agg_plain["cached"])
+            if gp["launches"]:
+                rows_ms = sum(a["ms"] for n, a in agg_plain["cached"].items() if n in ("resid_norm", "qkv_rope_scatter", "swiglu"))
+                tot_plain = sum(a["ms"] for a in agg_plain["cached"].values())
+                tot_fused = sum(a["ms"] for a in agg["cached"].values())
+                ach_p = gp["weight_bytes"] / (gp["ms"] * 1e-3) / 1e9
+                roofline["row_tails_as_kernels"] = {
+                    "achieved": ach_p, "frac": ach_p / pk["hbm"], "avg_launch_us": gp["ms"] * 1e3 / gp["launches"],
+                    "row_kernel_share_of_cached_steps": rows_ms / tot_plain if tot_plain else None,
+                    "cached_steps_event_ms": {"tails_fused": tot_fused, "tails_as_kernels": tot_plain},
+                    "what": "the same steps with DKV_FUSE_TAILS=0: GEMM launches hold the projection alone (weights "
+                            "only / launch time), the split-K reduction, residual, norm statistics, RoPE and scatter "
+                            "run as row kernels"}
         if gr["launches"]:
             ach = gr["flops"] / (gr["ms"] * 1e-3) / 1e12
             roofline_tensor = {"bound": "tensor", "kernel": "k_gemm_tc / k_gemm_tc2, launches of the refresh steps "
