@@ -278,6 +278,27 @@ int dkv_status(dkv_cache* cache, int32_t* word);
  * [batch][kv_head][pos][head_dim] in the activation type. */
 int dkv_cache_slots(const dkv_cache* cache, int layer, void** k_slots, void** v_slots);
 
+/* Checkpoint / resume of a generation.  What Algorithm 1 carries from one
+ * step to the next is the cached Key and Value states and the previous step's
+ * sets (M_{t-1} for Eq. 4, D_{t-1} for the window rule of Sec. 3.4); together
+ * with the step / refresh counters, the provenance stamps and the statistics
+ * that is the whole state of a handle between two dkv_step calls.
+ * dkv_cache_export copies it into `state_host` (HOST memory, at least
+ * dkv_cache_state_bytes() bytes: a fixed header, then the K/V slots of every
+ * layer and the stored sets); dkv_cache_import loads such a blob into a live
+ * handle of the SAME model geometry, batch, seq_len, prompt_len, max_k and
+ * policy (on any device, with its own arena), after which dkv_step continues
+ * exactly where the exporting handle stood: same active rows, refresh
+ * schedule and results.  The caller's tokens / masked arrays are not part of
+ * the state.  Both calls synchronise `stream` (and the stream of the handle's
+ * last step) before they return.  The blob is valid for this library version
+ * only.  Errors: INVALID_ARG (NULL, not an exported state, counters out of
+ * range), NOMEM (export: state_bytes too small), SHAPE (import: geometry or
+ * policy differ, truncated blob), STATE, CUDA. */
+size_t dkv_cache_state_bytes(const dkv_cache* cache);
+int dkv_cache_export(dkv_cache* cache, void* state_host, size_t state_bytes, void* stream);
+int dkv_cache_import(dkv_cache* cache, const void* state_host, size_t state_bytes, void* stream);
+
 /* Per-kernel-class timing: when enabled, every launch is bracketed by CUDA
  * events on the launching stream (this slows a step slightly; not for timed
  * throughput runs).  dkv_profile_read synchronises and returns, per class, the

@@ -30,6 +30,7 @@ EXPORTS = [
     "dkv_get_stats", "dkv_get_provenance", "dkv_get_index_maps", "dkv_status", "dkv_cache_slots",
     "dkv_profile_enable", "dkv_profile_read", "dkv_gemm_workspace_bytes", "dkv_op_gemm", "dkv_op_attention",
     "dkv_static_scratch_bytes", "dkv_op_gemm_static", "dkv_trace_set", "dkv_debug_tail_wait",
+    "dkv_cache_state_bytes", "dkv_cache_export", "dkv_cache_import",
 ]
 
 
@@ -105,6 +106,10 @@ def load():
     lib.dkv_get_index_maps.argtypes = [vp, vp, vp, vp, vp]
     lib.dkv_status.argtypes = [vp, C.POINTER(C.c_int32)]
     lib.dkv_cache_slots.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp)]
+    lib.dkv_cache_state_bytes.restype = sz
+    lib.dkv_cache_state_bytes.argtypes = [vp]
+    lib.dkv_cache_export.argtypes = [vp, vp, sz, vp]
+    lib.dkv_cache_import.argtypes = [vp, vp, sz, vp]
     lib.dkv_profile_enable.argtypes = [vp, i32]
     lib.dkv_profile_read.argtypes = [vp, C.POINTER(dkv_profile_entry), C.POINTER(C.c_int)]
     lib.dkv_gemm_workspace_bytes.restype = sz
@@ -118,7 +123,7 @@ def load():
     lib.dkv_op_gemm_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
     for name in EXPORTS:
         if name not in ("dkv_strerror", "dkv_model_bytes", "dkv_cache_bytes", "dkv_gemm_workspace_bytes",
-                        "dkv_static_scratch_bytes"):
+                        "dkv_static_scratch_bytes", "dkv_cache_state_bytes"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -300,6 +305,21 @@ def dkv_cache_slots(cache: Cache, layer: int):
     k, v = C.c_void_p(), C.c_void_p()
     _check("dkv_cache_slots", load().dkv_cache_slots(cache.handle, layer, C.byref(k), C.byref(v)))
     return k.value, v.value
+
+
+def dkv_cache_state_bytes(cache: Cache) -> int:
+    return load().dkv_cache_state_bytes(cache.handle)
+
+
+def dkv_cache_export(cache: Cache, state_host, stream=None):
+    """state_host: a CPU uint8 tensor of at least dkv_cache_state_bytes(cache) bytes."""
+    _check("dkv_cache_export", load().dkv_cache_export(cache.handle, _ptr(state_host), state_host.numel(),
+                                                       _stream(stream)))
+
+
+def dkv_cache_import(cache: Cache, state_host, stream=None):
+    _check("dkv_cache_import", load().dkv_cache_import(cache.handle, _ptr(state_host), state_host.numel(),
+                                                       _stream(stream)))
 
 
 def dkv_profile_enable(cache: Cache, on: bool):

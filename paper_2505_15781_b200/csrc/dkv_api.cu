@@ -1539,6 +1539,164 @@ int dkv_cache_slots(const dkv_cache* c, int layer, void** k_slots, void** v_slot
   return DKV_OK;
 }
 
+// ---------------------------------------------------- state export / import
+namespace {
+
+constexpr uint64_t STATE_MAGIC = 0x314554415453564bull;   // "KVSTATE1", little-endian
+constexpr uint32_t STATE_VERSION = 1;
+
+// Header of an exported state; the device sections follow in the order of state_sections().
+struct StateHeader {
+  uint64_t magic;
+  uint32_t version, header_bytes;
+  int64_t total_bytes;
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, dtype, act_dtype, elem_bytes;
+  int32_t B, L, P, kmax;
+  dkv_policy policy;
+  int32_t step, last_refresh, pending_refresh, prev_rows_bound, have_dprev, prev_k;
+  dkv_stats stats;
+  uint64_t active_rows_dev;   // the device-side count of active rows
+};
+
+struct StateSection {
+  void* dev;
+  size_t bytes;
+};
+
+// What a later step reads from earlier ones: the K/V slots, both stored mask sets, both stored D
+// sets and the provenance stamps.
+int state_sections(const dkv_cache* c, StateSection* out /*[7]*/) {
+  const Arena& a = c->ar;
+  const dkv_model_desc& md = c->model->desc;
+  const size_t BL = static_cast<size_t>(c->dims.B) * c->dims.L;
+  const size_t slots = static_cast<size_t>(md.n_layers) * c->dims.B * md.n_kv_heads * c->dims.L * md.head_dim * c->model->asize;
+  const size_t dset = static_cast<size_t>(c->dims.B) * c->dims.kmax * 4;
+  out[0] = {a.k_slots, slots};
+  out[1] = {a.v_slots, slots};
+  out[2] = {a.mask_buf[0], BL};
+  out[3] = {a.mask_buf[1], BL};
+  out[4] = {a.d_buf[0], dset};
+  out[5] = {a.d_buf[1], dset};
+  out[6] = {a.written_step, BL * 4};
+  return 7;
+}
+
+size_t state_total(const dkv_cache* c) {
+  StateSection sec[7];
+  const int n = state_sections(c, sec);
+  size_t total = align_up(sizeof(StateHeader), 256);
+  for (int i = 0; i < n; ++i) total += align_up(sec[i].bytes, 256);
+  return total;
+}
+
+void state_fill_geometry(const dkv_cache* c, StateHeader* h) {
+  const dkv_model_desc& md = c->model->desc;
+  h->n_layers = md.n_layers;
+  h->d_model = md.d_model;
+  h->n_q_heads = md.n_q_heads;
+  h->n_kv_heads = md.n_kv_heads;
+  h->head_dim = md.head_dim;
+  h->dtype = md.dtype;
+  h->act_dtype = md.act_dtype;
+  h->elem_bytes = static_cast<int32_t>(c->model->asize);
+  h->B = c->dims.B;
+  h->L = c->dims.L;
+  h->P = c->dims.P;
+  h->kmax = c->dims.kmax;
+  h->policy = c->policy;
+}
+
+}  // namespace
+
+size_t dkv_cache_state_bytes(const dkv_cache* c) {
+  if (!c || !live_cache(c)) return 0;
+  return state_total(c);
+}
+
+int dkv_cache_export(dkv_cache* c, void* state_host, size_t state_bytes, void* stream) {
+  if (!c || !state_host) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
+  const size_t total = state_total(c);
+  if (state_bytes < total) return DKV_E_NOMEM;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the steps so far may have run on another stream
+  if (c->last_stream != st && cudaStreamSynchronize(c->last_stream) != cudaSuccess) return DKV_E_CUDA;
+  uint8_t* dst = static_cast<uint8_t*>(state_host);
+  StateHeader h;
+  memset(&h, 0, sizeof(h));
+  h.magic = STATE_MAGIC;
+  h.version = STATE_VERSION;
+  h.header_bytes = static_cast<uint32_t>(align_up(sizeof(StateHeader), 256));
+  h.total_bytes = static_cast<int64_t>(total);
+  state_fill_geometry(c, &h);
+  h.step = c->step;
+  h.last_refresh = c->last_refresh;
+  h.pending_refresh = c->pending_refresh;
+  h.prev_rows_bound = c->prev_rows_bound;
+  h.have_dprev = c->have_dprev ? 1 : 0;
+  h.prev_k = c->prev_k;
+  h.stats = c->stats;
+  StateSection sec[7];
+  const int n = state_sections(c, sec);
+  size_t off = h.header_bytes;
+  for (int i = 0; i < n; ++i) {
+    if (cudaMemcpyAsync(dst + off, sec[i].dev, sec[i].bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DKV_E_CUDA;
+    off += align_up(sec[i].bytes, 256);
+  }
+  if (cudaMemcpyAsync(&h.active_rows_dev, c->ar.status + 2, 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DKV_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DKV_E_CUDA;
+  memset(dst, 0, h.header_bytes);
+  memcpy(dst, &h, sizeof(h));
+  return DKV_OK;
+}
+
+int dkv_cache_import(dkv_cache* c, const void* state_host, size_t state_bytes, void* stream) {
+  if (!c || !state_host) return DKV_E_INVALID_ARG;
+  DKV_CHECK_CACHE(c);
+  if (state_bytes < sizeof(StateHeader)) return DKV_E_INVALID_ARG;
+  StateHeader h;
+  memcpy(&h, state_host, sizeof(h));
+  if (h.magic != STATE_MAGIC || h.version != STATE_VERSION) return DKV_E_INVALID_ARG;
+  StateHeader want;
+  memset(&want, 0, sizeof(want));
+  state_fill_geometry(c, &want);
+  if (h.n_layers != want.n_layers || h.d_model != want.d_model || h.n_q_heads != want.n_q_heads ||
+      h.n_kv_heads != want.n_kv_heads || h.head_dim != want.head_dim || h.dtype != want.dtype ||
+      h.act_dtype != want.act_dtype || h.elem_bytes != want.elem_bytes || h.B != want.B || h.L != want.L ||
+      h.P != want.P || h.kmax != want.kmax || memcmp(&h.policy, &want.policy, sizeof(dkv_policy)) != 0)
+    return DKV_E_SHAPE;
+  const size_t total = state_total(c);
+  if (h.total_bytes != static_cast<int64_t>(total) || h.header_bytes != align_up(sizeof(StateHeader), 256) ||
+      state_bytes < total)
+    return DKV_E_SHAPE;
+  if (h.step < 0 || h.last_refresh < 0 || h.pending_refresh < -1 || h.pending_refresh > DKV_REFRESH_DECODED_ONLY ||
+      h.prev_rows_bound < 0 || h.prev_rows_bound > want.L || h.prev_k < 0 || h.prev_k > want.kmax)
+    return DKV_E_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (c->last_stream != st && cudaStreamSynchronize(c->last_stream) != cudaSuccess) return DKV_E_CUDA;
+  const uint8_t* src = static_cast<const uint8_t*>(state_host);
+  StateSection sec[7];
+  const int n = state_sections(c, sec);
+  size_t off = h.header_bytes;
+  for (int i = 0; i < n; ++i) {
+    if (cudaMemcpyAsync(sec[i].dev, src + off, sec[i].bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return DKV_E_CUDA;
+    off += align_up(sec[i].bytes, 256);
+  }
+  if (cudaMemcpyAsync(c->ar.status + 2, &h.active_rows_dev, 8, cudaMemcpyHostToDevice, st) != cudaSuccess) return DKV_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DKV_E_CUDA;
+  c->step = h.step;
+  c->last_refresh = h.last_refresh;
+  c->pending_refresh = h.pending_refresh;
+  c->prev_rows_bound = h.prev_rows_bound;
+  c->have_dprev = h.have_dprev != 0;
+  c->prev_k = h.prev_k;
+  const int64_t launches = c->stats.kernel_launches;
+  c->stats = h.stats;
+  c->stats.kernel_launches = launches;   // launches are this handle's own
+  c->last_stream = st;
+  return DKV_OK;
+}
+
 int dkv_profile_enable(dkv_cache* c, int on) {
   DKV_CHECK_CACHE(c);
   if (!on && c->profiling) prof_flush(c);

@@ -55,6 +55,10 @@ def test_a_handle_that_is_not_live_is_a_state_error():
     assert lib.dkv_get_index_maps(bogus, None, None, None, None) == -3
     assert lib.dkv_cache_slots(bogus, 0, None, None) == -3
     assert lib.dkv_profile_enable(bogus, 1) == -3
+    assert lib.dkv_cache_state_bytes(bogus) == 0
+    assert lib.dkv_cache_export(bogus, one, 4096, None) == -3
+    assert lib.dkv_cache_import(bogus, one, 4096, None) == -3
+    assert lib.dkv_cache_export(None, one, 4096, None) == -1
     assert lib.dkv_cache_destroy(bogus) == -3
     assert lib.dkv_model_destroy(bogus) == -3
     assert lib.dkv_cache_bytes(bogus, 1, 16, None) == 0
