@@ -543,6 +543,7 @@ struct HeadStats {   // vocabulary-head mode of the GEMM epilogue
   int* st_arg;
   float* st_m2;   // NULL unless the score needs the second maximum / the entropy sum
   float* st_t;
+  mutable int n_groups = 0;   // out: entries per row the launch writes (4 per CTA)
 };
 
 // Per-row scale of a GEMM's result: the RMSNorm of its operand, applied after the product.
@@ -681,6 +682,11 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
   p.st_t = o.head ? o.head->st_t : nullptr;
   const int sms = sm_count();
   const int grid = std::min(p.units, sms);
+  if (o.head) {
+    // a CTA keeps the statistics of one row tile across its weight tiles
+    if (p.r_tiles != 1 || splits != 1) return DKV_E_SHAPE;
+    o.head->n_groups = 4 * grid;
+  }
   // the CTAs of a tile wait for each other in the fused tail: every unit needs a resident CTA of its own
   if (o.tail.mode != FUSE_NONE && p.units <= sms && p.units <= MAX_TILE_COUNTERS) {
     const FusedTail& t = o.tail;
@@ -978,15 +984,21 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     head_sc.d = d;
   }
   // 16-bit modes, no logits requested: the head GEMM's epilogue reduces every 32 token ids to
-  // (max, argmax, sum exp) with warp shuffles and a small kernel combines them; the logits are
-  // never written.  Otherwise (check mode, or the caller wants the logits) they are materialised.
+  // (max, argmax, sum exp) with warp shuffles, joins them over the weight tiles of a CTA, and a small
+  // kernel combines the CTAs' entries; the logits are never written.  Otherwise (check mode, or the caller wants the logits) they are materialised.
   // (the warp-shuffle reduction costs time in proportion to the head rows: with many of them the
   // GEMM is compute-bound and writing the logits is the cheaper way)
   if (bf16 && !logits_dbg && H <= 128) {
     int splits;
     long long stride;
     const int score = c->policy.score;
-    HeadStats hs = {md.mask_id, a.st_max, a.st_sum, a.st_arg, score ? a.st_m2 : nullptr, score ? a.st_t : nullptr};
+    HeadStats hs;
+    hs.mask_id = md.mask_id;
+    hs.st_max = a.st_max;
+    hs.st_sum = a.st_sum;
+    hs.st_arg = a.st_arg;
+    hs.st_m2 = score ? a.st_m2 : nullptr;
+    hs.st_t = score ? a.st_t : nullptr;
     {
       const double bytes = (static_cast<double>(md.vocab) * d + static_cast<double>(H) * d) * es;
       Launch lk(c, st, PC_GEMM_HEAD, bytes, 2.0 * H * md.vocab * static_cast<double>(d));
@@ -998,14 +1010,14 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
                    &splits, &stride, o);
       if (rc) return rc;
     }
-    Launch lk(c, st, PC_HEAD_STATS, 24.0 * H * ((md.vocab + 31) / 32), 0);
+    Launch lk(c, st, PC_HEAD_STATS, 24.0 * H * hs.n_groups, 0);
     static PerDeviceOnce comb_once;
     if (comb_once.need() &&
         cudaFuncSetAttribute(k_head_combine, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024) != cudaSuccess)
       return DKV_E_CUDA;
     launch_k(k_head_combine, H, 256, 100 * 1024, st, static_cast<const float*>(a.st_max), static_cast<const float*>(a.st_sum),
              static_cast<const int*>(a.st_arg), static_cast<const float*>(a.st_m2), static_cast<const float*>(a.st_t),
-             score, (md.vocab + 31) / 32, H, h_dev, a.head_pos, conf, pred);
+             score, hs.n_groups, H, h_dev, a.head_pos, conf, pred);
     return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
   }
   float* logits = logits_dbg ? logits_dbg : a.logits;

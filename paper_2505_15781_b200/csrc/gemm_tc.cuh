@@ -37,6 +37,7 @@
 // one unit per CTA is a dependent chain of tensor-memory loads and stores per
 // warp; eight warps halve it).
 #pragma once
+#include "head_stat.cuh"
 #include "pdl.cuh"
 #include "ptx.cuh"
 
@@ -115,7 +116,7 @@ struct GemmTcParams {
   // rows (= 32 token ids) and every row r, the largest logit, its id and sum exp(logit - max)
   int head_mode;
   int mask_id;             // token id left out of the statistics
-  float* st_max;           // [ceil(n / 32)][r_bound]
+  float* st_max;           // [4 * gridDim.x][r_bound]: per CTA and lane quarter, over all its weight tiles
   float* st_sum;
   int* st_arg;
   float* st_m2;            // second largest logit of the 32 ids (scores other than the max probability)
@@ -468,6 +469,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     if (trace_on() && threadIdx.x == 64) trace_store(3, t_enter);
     int r_valid = p.r_bound;
     if (p.r_dev) r_valid = min(r_valid, *p.r_dev);
+    // head mode: the statistics of this warp's token ids over ALL weight tiles of the CTA, per row
+    // (lane l < 16 keeps row cs * 16 + 32 * i + l in run<i>); written once after the last tile
+    HeadStat run0 = head_stat_empty(), run1 = run0, run2 = run0, run3 = run0;
     int j = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++j) {
@@ -560,7 +564,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           if (p.head_mode) {
             // softmax statistics over this warp's 32 token ids, per row, by warp shuffles
             const bool live = n < p.n && n != p.mask_id;
-            const long long slot = static_cast<long long>((n0 + h * GEMM_BM) / 32 + q) * p.r_bound;
+            HeadStat mine = head_stat_empty();
 #pragma unroll
             for (int jj = 0; jj < 16; ++jj) {
               const float val = live ? __uint_as_float(v[jj]) : -INFINITY;
@@ -590,17 +594,20 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                   tt += __shfl_xor_sync(0xffffffffu, tt, o);
                 }
               }
-              const int r = r0 + c + jj;
-              if (lane == jj && r < r_valid) {
-                p.st_max[slot + r] = m;
-                p.st_sum[slot + r] = e;
-                p.st_arg[slot + r] = arg;
-                if (p.st_m2) {
-                  p.st_m2[slot + r] = m2;
-                  p.st_t[slot + r] = tt;
-                }
+              if (lane == jj) {      // lane jj keeps row c + jj
+                mine.m = m;
+                mine.s = e;
+                mine.arg = arg;
+                mine.m2 = m2;
+                mine.t = tt;
               }
             }
+            // joined with what this warp has seen of the row in earlier weight tiles
+            const int ci = c >> 5;
+            if (ci == 0) run0 = head_stat_merge(run0, mine);
+            else if (ci == 1) run1 = head_stat_merge(run1, mine);
+            else if (ci == 2) run2 = head_stat_merge(run2, mine);
+            else run3 = head_stat_merge(run3, mine);
           } else if (n < p.n) {
             float* dst = out + static_cast<long long>(r0 + c) * p.ldo + n;
             if (r0 + c + 16 <= r_valid) {           // whole group valid: no per-row test
@@ -650,6 +657,24 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
         if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
         else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
+      }
+    }
+    if (p.head_mode && ok && lane < 16) {
+      // one entry per (CTA, lane quarter) and row: arrays [gridDim.x * 4][r_bound] (one row tile)
+      const long long at = static_cast<long long>(blockIdx.x * 4 + q) * p.r_bound;
+#pragma unroll
+      for (int ci = 0; ci < 4; ++ci) {
+        const HeadStat& r = ci == 0 ? run0 : ci == 1 ? run1 : ci == 2 ? run2 : run3;
+        const int row = cs * 16 + 32 * ci + lane;
+        if (row < r_valid) {
+          p.st_max[at + row] = r.m;
+          p.st_sum[at + row] = r.s;
+          p.st_arg[at + row] = r.arg;
+          if (p.st_m2) {
+            p.st_m2[at + row] = r.m2;
+            p.st_t[at + row] = r.t;
+          }
+        }
       }
     }
   }

@@ -9,6 +9,7 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+#include "head_stat.cuh"
 #include "pdl.cuh"
 
 namespace dkv {
@@ -489,53 +490,8 @@ k_head_stats(const float* __restrict__ logits, const int* __restrict__ n_head_de
   }
 }
 
-// Softmax statistics of a set of token ids: the largest logit m (its id: lowest on ties), the second
-// largest m2 (over the other ids), S = sum exp(l - m) and T = sum exp(l - m)(l - m).  merge() joins the
-// statistics of two disjoint sets; it is exact in (m, arg, m2) and order-independent there.
-struct HeadStat {
-  float m, m2, s, t;
-  int arg;
-};
-__device__ __forceinline__ HeadStat head_stat_empty() {
-  HeadStat e;
-  e.m = -CUDART_INF_F;
-  e.m2 = -CUDART_INF_F;
-  e.s = 0.f;
-  e.t = 0.f;
-  e.arg = 0x7fffffff;
-  return e;
-}
-__device__ __forceinline__ HeadStat head_stat_merge(const HeadStat& a, const HeadStat& b) {
-  const bool b_wins = b.m > a.m || (b.m == a.m && b.arg < a.arg);
-  const HeadStat& hi = b_wins ? b : a;
-  const HeadStat& lo = b_wins ? a : b;
-  HeadStat r;
-  r.m = hi.m;
-  r.arg = hi.arg;
-  r.m2 = fmaxf(fmaxf(hi.m2, lo.m2), lo.m);
-  if (lo.m == -CUDART_INF_F) {          // an empty side (also when both are empty): nothing to rescale
-    r.s = hi.s;
-    r.t = hi.t;
-  } else {
-    const float dm = lo.m - hi.m;        // <= 0
-    const float w = expf(dm);
-    r.s = hi.s + w * lo.s;
-    r.t = hi.t + w * (lo.t + lo.s * dm);
-  }
-  return r;
-}
-__device__ __forceinline__ HeadStat head_stat_shfl_xor(const HeadStat& v, int o) {
-  HeadStat r;
-  r.m = __shfl_xor_sync(0xffffffffu, v.m, o);
-  r.m2 = __shfl_xor_sync(0xffffffffu, v.m2, o);
-  r.s = __shfl_xor_sync(0xffffffffu, v.s, o);
-  r.t = __shfl_xor_sync(0xffffffffu, v.t, o);
-  r.arg = __shfl_xor_sync(0xffffffffu, v.arg, o);
-  return r;
-}
-
-// Combine the per-32-id statistics of the head GEMM (arrays [ceil(V/32)][ld], one column per head row):
-// one pass per head row with an online merge per thread, then a merge across the block; the score is
+// Combine the statistics the head GEMM left per CTA and lane quarter (arrays [n_groups][ld], one column
+// per head row): one pass per head row with an online merge per thread, then a merge across the block; the score is
 // written at the row's original position.  One CTA of 256 threads per row.  The launch asks for enough
 // dynamic shared memory that an SM holds one block: launched early behind the head GEMM, the blocks would
 // otherwise pile up on the few SMs with room and run several times longer.
