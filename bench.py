@@ -56,7 +56,7 @@ WORKLOADS = {
 # DRAM traffic (read + write) per launch of the projection GEMMs: a RECORDED constant from the ncu capture
 # summarised in profiles/k_gemm_tc_llada8b_decode_2layers.md (256 active rows; per launch, independent of
 # depth), not measured by this run.
-NCU_GEMM_TRAFFIC = {"gemm_qkv": 106.7e6, "gemm_o": 41.3e6, "gemm_gateup": 207.0e6, "gemm_down": 115.3e6}
+NCU_GEMM_TRAFFIC = {"gemm_qkv": 106.8e6, "gemm_o": 41.4e6, "gemm_gateup": 206.8e6, "gemm_down": 114.7e6}
 NCU_GEMM_TRAFFIC_SOURCE = "ncu capture summarised in profiles/k_gemm_tc_llada8b_decode_2layers.md (recorded constant)"
 
 
