@@ -138,6 +138,21 @@ def test_medium_widths_split_k_with_and_without_fused_tails(ms, pol, k, fuse, mo
     assert worst < BF16_TOL_SIGMA
 
 
+@pytest.mark.parametrize("fuse", [1, 0])
+@pytest.mark.parametrize("ms,pol,k,batch,P", [(MEDIUM_128, O.Policy(O.POLICY_DECODE, 2), 2, 3, 84),
+                                              (MEDIUM_64, O.Policy(O.POLICY_PD, 3), 3, 4, 70),
+                                              (MEDIUM_64, O.Policy(O.POLICY_NONE), 2, 3, 90),
+                                              (MEDIUM_128, O.Policy(O.POLICY_PREFILL, isolated_prefill=True), 2, 5, 60)])
+def test_medium_widths_more_than_one_row_tile(ms, pol, k, batch, P, fuse, monkeypatch):
+    """Full and refresh steps with more than 256 active rows over several sequences (several row tiles
+    per projection, the row kernels behind the multi-tile launches, sequence index and position of
+    every row in RoPE and the slot scatter), with the fused tails of the cached steps on and off;
+    head_dim 64 and 128, GQA, both head paths, against the oracle."""
+    monkeypatch.setenv("DKV_FUSE_TAILS", str(fuse))
+    worst = run_forced(ms, True, batch, P, 6 * k, k, pol, None, seed=9)
+    assert worst < BF16_TOL_SIGMA
+
+
 def free_run(ms, bf16, batch, P, G, k, pol, block, seed=0, host=False):
     W, model = U.build_pair(ms, seed, bf16)
     prompts = synth.make_prompt(batch, P, min(1000, ms.vocab - 1), seed)
