@@ -113,6 +113,26 @@ int make_tmap(CUtensorMap* tm, const void* base, long long rows, long long k, in
   return r == CUDA_SUCCESS ? DKV_OK : DKV_E_CUDA;
 }
 
+// Tensor map of a weight matrix stored in blocks of 128 rows x 64 columns ([ceil(rows / 128)][ceil(k / 64)]
+// blocks of 16 KB each, zero-padded): the box the GEMM loads per weight half and k-block is then one
+// contiguous piece of memory instead of 128 pieces of 128 bytes a row pitch apart.
+int make_tmap_blocked(CUtensorMap* tm, const void* base, long long rows, long long k) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return DKV_E_CUDA;
+  const long long blocks = ((rows + GEMM_BM - 1) / GEMM_BM) * ((k + GEMM_BK - 1) / GEMM_BK);
+  cuuint64_t gdim[2] = {static_cast<cuuint64_t>(GEMM_BK), static_cast<cuuint64_t>(blocks * GEMM_BM)};
+  cuuint64_t gstride[1] = {static_cast<cuuint64_t>(GEMM_BK) * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(GEMM_BK), static_cast<cuuint32_t>(GEMM_BM)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? DKV_OK : DKV_E_CUDA;
+}
+inline size_t blocked_bytes(long long rows, long long k) {
+  return static_cast<size_t>((rows + GEMM_BM - 1) / GEMM_BM) * ((k + GEMM_BK - 1) / GEMM_BK) * GEMM_BM * GEMM_BK * 2;
+}
+
 // 16-bit tensor with 128-byte rows of 64 elements innermost, up to 3 dimensions (dims / box innermost
 // first, strides in bytes for dimensions 1..rank-1), 128-byte swizzle.
 int make_tmap_nd(CUtensorMap* tm, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
@@ -222,6 +242,7 @@ struct dkv_model {
   int d_q, d_kv, n_qkv;
   size_t esize;   // bytes per weight element
   size_t asize;   // bytes per activation / cache element
+  bool w_blocked; // the layers' fp16 weight copies are stored in 128 x 64 blocks (make_tmap_blocked)
   int gu_blk;     // 128: the gate/up copy is regrouped [128 gate | 128 up] per 256 rows (SwiGLU in the GEMM epilogue); 0: not
   bool gu_pair;   // the standalone SwiGLU launch runs on CTA pairs (d_ffn a multiple of 256)
 };
@@ -577,6 +598,7 @@ struct FusedTail {
 struct GemmOpts {
   int forced_splits = 0;
   bool w_static = true;
+  bool w_blocked = false;                    // tw is a make_tmap_blocked map
   const HeadStats* head = nullptr;
   void* swiglu_out = nullptr;
   int ld_u = 0;
@@ -611,6 +633,7 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
   p.status = status;
   p.x_bf16 = x_bf16 ? 1 : 0;
   p.w_static = o.w_static ? 1 : 0;
+  p.w_blocked = o.w_blocked ? 1 : 0;
   p.swiglu_out = o.swiglu_out;
   p.ld_u = o.ld_u;
   p.mask_id = -1;
@@ -826,7 +849,11 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     const double bytes = (static_cast<double>(n) * k + static_cast<double>(rb) * k) * es + 4.0 * rb * n;
     Launch l(c, st, cls, bytes, 2.0 * rb * n * static_cast<double>(k));
     if (fused) *fused = false;
-    if (bf16) return gemm_tc(*tw, c->xmaps[xb], n, k, rb, rdev, out, dm.part_rows, a.status, x_bf16, st, splits, stride, o, fused);
+    if (bf16) {
+      GemmOpts ob = o;
+      ob.w_blocked = m->w_blocked;
+      return gemm_tc(*tw, c->xmaps[xb], n, k, rb, rdev, out, dm.part_rows, a.status, x_bf16, st, splits, stride, ob, fused);
+    }
     *splits = 1;
     *stride = 0;
     return gemm_f32(static_cast<const float*>(x), static_cast<const float*>(w), n, k, rb, rdev, out, st);
@@ -954,6 +981,7 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       o.ld_u = f;
       o.xmaps_half = m->gu_pair ? c->xmaps_half : nullptr;
       o.row_tiles = R > 256 ? gu_rt : 0;
+      o.w_blocked = m->w_blocked;
       rc = gemm_tc(lm->wgu, c->xmaps[XB_XN], 2 * f, d, R, r_dev, a.part, dm.part_rows, a.status, x_bf16, st, &splits,
                    &stride, o);
       if (rc) return rc;
@@ -1201,7 +1229,8 @@ size_t dkv_model_bytes(const dkv_model_desc* desc) {
   const size_t dq = static_cast<size_t>(desc->n_q_heads) * desc->head_dim;
   const size_t dkv = static_cast<size_t>(desc->n_kv_heads) * desc->head_dim;
   size_t per_layer = 0;
-  for (size_t n : {(dq + 2 * dkv) * d, d * dq, 2 * f * d, d * f}) per_layer += align_up(n * 2, 256);
+  per_layer += align_up(blocked_bytes(dq + 2 * dkv, d), 256) + align_up(blocked_bytes(d, dq), 256) +
+               align_up(blocked_bytes(2 * f, d), 256) + align_up(blocked_bytes(d, f), 256);
   return per_layer * desc->n_layers + align_up(static_cast<size_t>(desc->vocab) * d * 2, 256) + 256;
 }
 
@@ -1255,27 +1284,27 @@ int dkv_model_create(const dkv_model_desc* desc, const dkv_weights* w, void* are
     };
     m->gu_blk = (f16 && desc->d_ffn % 128 == 0) ? 128 : 0;
     m->gu_pair = m->gu_blk && desc->d_ffn % 256 == 0;
+    m->w_blocked = f16;
     m->maps.resize(desc->n_layers);
     int rc = DKV_OK;
     const long long d = desc->d_model, f = desc->d_ffn;
+    // fp16 mode: the layers' matrices are copied into 128 x 64 blocks (gate/up regrouped on the way);
+    // bf16 activations: the caller's row-major matrices are read in place
+    auto layer_map = [&](CUtensorMap* tm, const void* src, long long rows, long long k, int gu_f, int gu_blk) -> int {
+      if (!f16) return make_tmap(tm, src, rows, k, GEMM_BM, false);
+      __half* dst = reinterpret_cast<__half*>(cur);
+      cur += align_up(blocked_bytes(rows, k), 256);
+      dim3 grid(static_cast<unsigned>(ceil_div(static_cast<int>(k), GEMM_BK)), static_cast<unsigned>(ceil_div(static_cast<int>(rows), GEMM_BM)));
+      k_block_f16<<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(src), dst, static_cast<int>(rows),
+                                        static_cast<int>(k), gu_f, gu_blk);
+      return make_tmap_blocked(tm, dst, rows, k);
+    };
     for (int l = 0; l < desc->n_layers && rc == DKV_OK; ++l) {
       const dkv_layer_weights& lw = m->layers[l];
-      rc = make_tmap(&m->maps[l].wqkv, prep(lw.wqkv, m->n_qkv * d), m->n_qkv, d, GEMM_BM, f16);
-      if (!rc) rc = make_tmap(&m->maps[l].wo, prep(lw.wo, d * m->d_q), d, m->d_q, GEMM_BM, f16);
-      if (!rc) {
-        const void* wgu = lw.wgu;
-        if (m->gu_blk) {
-          __half* dst = reinterpret_cast<__half*>(cur);
-          cur += align_up(static_cast<size_t>(2 * f * d) * 2, 256);
-          k_gu_interleave_f16<<<static_cast<unsigned>(2 * f), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(lw.wgu), dst,
-                                                                          static_cast<int>(f), static_cast<int>(d), m->gu_blk);
-          wgu = dst;
-        } else {
-          wgu = prep(lw.wgu, 2 * f * d);
-        }
-        rc = make_tmap(&m->maps[l].wgu, wgu, 2 * f, d, GEMM_BM, f16);
-      }
-      if (!rc) rc = make_tmap(&m->maps[l].wd, prep(lw.wd, d * f), d, f, GEMM_BM, f16);
+      rc = layer_map(&m->maps[l].wqkv, lw.wqkv, m->n_qkv, d, 0, 0);
+      if (!rc) rc = layer_map(&m->maps[l].wo, lw.wo, d, m->d_q, 0, 0);
+      if (!rc) rc = layer_map(&m->maps[l].wgu, lw.wgu, 2 * f, d, static_cast<int>(f), m->gu_blk);
+      if (!rc) rc = layer_map(&m->maps[l].wd, lw.wd, d, f, 0, 0);
     }
     if (!rc) rc = make_tmap(&m->head_map, prep(m->head, static_cast<size_t>(desc->vocab) * d), desc->vocab, d, GEMM_BM, f16);
     if (!rc && cudaGetLastError() != cudaSuccess) rc = DKV_E_CUDA;

@@ -121,6 +121,7 @@ struct GemmTcParams {
   int* st_arg;
   float* st_m2;            // second largest logit of the 32 ids (scores other than the max probability)
   float* st_t;             // sum exp(l - max)(l - max)
+  int w_blocked;           // 1: tm_w maps a copy stored in 128 x 64 blocks, [ceil(n / 128)][kb_total] of them
   int w_static;            // 1: the weights were complete long before this launch, so they may be
                            // fetched before the wait on the stream predecessor
   // per-row scale of the result: NULL = none; rs_parts > 0: rs_src is [rs_parts][rs_ld] partial sums of
@@ -386,7 +387,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         mbar_expect_tx(full, static_cast<uint32_t>(p.stage_bytes));
         const uint32_t a_dst = smem_base + s * p.stage_bytes;
         for (int h = 0; h < p.halves; ++h)
-          tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, (c.kb0 + c.i) * GEMM_BK, c.n0 + h * GEMM_BM, pol_w);
+          if (p.w_blocked)      // block (row block, k-block) of a blocked copy: rows block * 128 .. + 127 of its map
+            tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, 0,
+                             (c.n0 + h * GEMM_BM) * p.kb_total + (c.kb0 + c.i) * GEMM_BM, pol_w);
+          else
+            tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, (c.kb0 + c.i) * GEMM_BK, c.n0 + h * GEMM_BM, pol_w);
       };
       auto load_b = [&](const Cursor& c, int it) {
         const int s = it % STAGES;

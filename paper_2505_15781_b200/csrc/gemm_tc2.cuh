@@ -176,8 +176,13 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         const uint32_t lf = mapa_shared(smem_u32(&full[s]), 0);
         const uint32_t a_dst = smem_base + s * p.stage_bytes;
         for (int h = 0; h < 2; ++h)
-          tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, (c.kb0 + c.i) * GEMM_BK,
-                                c.n0 + static_cast<int>(rank) * 256 + h * GEMM_BM, pol_w);
+          if (p.w_blocked)
+            tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, 0,
+                                  (c.n0 + static_cast<int>(rank) * 256 + h * GEMM_BM) * p.kb_total +
+                                      (c.kb0 + c.i) * GEMM_BM, pol_w);
+          else
+            tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, (c.kb0 + c.i) * GEMM_BK,
+                                  c.n0 + static_cast<int>(rank) * 256 + h * GEMM_BM, pol_w);
       };
       auto load_b = [&](const Cursor& c, int it) {
         const int s = it % STAGES;

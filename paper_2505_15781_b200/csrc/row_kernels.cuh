@@ -51,26 +51,34 @@ __global__ void __launch_bounds__(256) k_bf16_to_f16(const __nv_bfloat16* __rest
     out[i] = __float2half_rn(__bfloat162float(in[i]));
 }
 
-// fp16 copy of the stacked [gate ; up] matrix with the rows regrouped as
-// [blk gate rows | blk up rows] per tile of 2 * blk rows (blk = 128: one CTA's tile, 256: a CTA
-// pair's), so that the GEMM epilogue finds gate_j and up_j of a feature in the two accumulators of
-// one thread.
-// grid: one CTA per destination row, 2f rows of d elements (d a multiple of 8).
-__global__ void __launch_bounds__(256) k_gu_interleave_f16(const __nv_bfloat16* __restrict__ in,
-                                                           __half* __restrict__ out, int f, int d, int blk) {
-  const int dst = blockIdx.x;
-  const int tile = dst / (2 * blk), half = (dst / blk) & 1, i = dst % blk;
-  const long long src = static_cast<long long>(half) * f + tile * blk + i;
-  const uint4* s = reinterpret_cast<const uint4*>(in + src * d);
-  uint4* o = reinterpret_cast<uint4*>(out + static_cast<long long>(dst) * d);
-  for (int c = threadIdx.x; c < d / 8; c += 256) {
-    const uint4 v = s[c];
-    const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
-    uint4 w;
-    __half2* h = reinterpret_cast<__half2*>(&w);
+// fp16 copy of a bf16 weight matrix [rows, k] in blocks of 128 rows x 64 columns, block (i, j) at
+// (i * ceil(k / 64) + j) * 8192 elements, rows inside a block 64 elements apart, zeros past the
+// matrix: what the projection GEMM loads per weight half and k-block is one contiguous 16 KB piece.
+// With gu_blk > 0 the matrix is [gate (gu_f rows); up (gu_f rows)] and the copy's rows are regrouped
+// [gu_blk gate rows | gu_blk up rows] per 2 * gu_blk, so that the GEMM epilogue finds gate_j and up_j
+// of a feature in the two accumulators of one thread.
+// grid (ceil(k / 64), ceil(rows / 128)), 256 threads; k a multiple of 8.
+__global__ void __launch_bounds__(256) k_block_f16(const __nv_bfloat16* __restrict__ in, __half* __restrict__ out,
+                                                   int rows, int k, int gu_f, int gu_blk) {
+  const long long blk = static_cast<long long>(blockIdx.y) * gridDim.x + blockIdx.x;
+  uint4* o = reinterpret_cast<uint4*>(out + blk * (128 * 64));
+  for (int e = threadIdx.x; e < 128 * 8; e += 256) {          // 8 vectors of 8 elements per row
+    const int r = e >> 3, c8 = e & 7;
+    const int dst = blockIdx.y * 128 + r, col = blockIdx.x * 64 + c8 * 8;
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (dst < rows && col < k) {
+      long long src = dst;
+      if (gu_blk > 0) {
+        const int tile = dst / (2 * gu_blk), half = (dst / gu_blk) & 1, i = dst % gu_blk;
+        src = static_cast<long long>(half) * gu_f + tile * gu_blk + i;
+      }
+      const uint4 v = *reinterpret_cast<const uint4*>(in + src * k + col);
+      const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
+      __half2* h = reinterpret_cast<__half2*>(&w);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) h[j] = __float22half2_rn(__bfloat1622float2(b[j]));
-    o[c] = w;
+      for (int j = 0; j < 4; ++j) h[j] = __float22half2_rn(__bfloat1622float2(b[j]));
+    }
+    o[e] = w;
   }
 }
 
