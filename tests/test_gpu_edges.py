@@ -202,6 +202,20 @@ def test_cache_slot_contents_match_the_oracles_cache(bf16):
             assert np.abs(g - ref).max() <= tol, f"layer {layer}: slot contents differ by {np.abs(g - ref).max()}"
 
 
+@pytest.mark.parametrize("ms", [synth.ModelShape(2, 328, 3, 3, 64, 344, 777, 776),      # nothing a multiple of 64
+                                synth.ModelShape(1, 200, 2, 1, 128, 136, 515, 514)])
+def test_widths_that_fill_neither_a_weight_block_nor_a_k_block(ms):
+    """d_model, d_ffn and the projections' row counts are multiples of 8 only: the last 64-column block
+    of every operand and the last 128-row block of every weight matrix are partly padding (zeros in the
+    blocked fp16 copies, the copy engine's fill for the row operands), and the vocabulary ends inside a
+    weight tile.  Full step, cached steps and a refresh against the oracle, both head paths."""
+    from tests.test_gpu_step import run_forced
+    worst = run_forced(ms, True, 2, 21, 12, 2, O.Policy(O.POLICY_DECODE, 3), 6, seed=13)
+    assert worst < 2e-2
+    worst = run_forced(ms, True, 3, 9, 8, 1, O.Policy(O.POLICY_PD, 0, isolated_prefill=True), None, seed=14)
+    assert worst < 2e-2
+
+
 def test_greedy_rejects_a_change_of_k_between_steps():
     """The window rule reads D_{t-1} with the k it was stored with."""
     ms = synth.tiny_shape()
