@@ -320,7 +320,60 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
   const int a_bytes = p.halves * GEMM_A_BYTES;
   const int tile_rows = p.halves * GEMM_BM;
 
+  // unit u -> (weight tile, row tile, split); consecutive units differ in the split first
+  auto decode = [&](int u, int& n0, int& r0, int& split, int& kb0, int& n_kb) {
+    split = u % p.splits;
+    const int t = u / p.splits;
+    r0 = (t % p.r_tiles) * p.br;
+    n0 = (t / p.r_tiles) * tile_rows;
+    kb0 = split * p.kb_per_split;
+    n_kb = max(0, min(p.kb_total, kb0 + p.kb_per_split) - kb0);
+  };
+
+  // The TMA producer (thread 0).  The weights never change, so the ring is first filled with weight
+  // tiles alone; only the activation rows have to wait for the kernel that produces them.  That first
+  // fill needs nothing but the producer's own barriers: it is issued before the CTA's set-up
+  // (tensor-memory allocation, the block-wide barrier) completes.
+  const uint64_t pol_w = l2_policy_evict_first();   // weights are streamed once per step
+  const uint64_t pol_x = l2_policy_evict_last();    // the few activation rows are re-read by every CTA
+  struct Cursor {
+    int u, i, n0, r0, split, kb0, n_kb;
+  } cur, head;
+  cur.u = blockIdx.x;
+  cur.i = 0;
+  auto settle = [&](Cursor& c) {   // move to the next k-block that exists (or past the end)
+    while (c.u < p.units) {
+      decode(c.u, c.n0, c.r0, c.split, c.kb0, c.n_kb);
+      if (c.i < c.n_kb) return true;
+      c.u += gridDim.x;
+      c.i = 0;
+    }
+    return false;
+  };
+  auto load_a = [&](const Cursor& c, int it) {
+    const int s = it % STAGES;
+    const uint32_t full = smem_u32(&bars[s]);
+    mbar_expect_tx(full, static_cast<uint32_t>(p.stage_bytes));
+    const uint32_t a_dst = smem_base + s * p.stage_bytes;
+    for (int h = 0; h < p.halves; ++h)
+      if (p.w_blocked)      // block (row block, k-block) of a blocked copy: rows block * 128 .. + 127 of its map
+        tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, 0,
+                         (c.n0 + h * GEMM_BM) * p.kb_total + (c.kb0 + c.i) * GEMM_BM, pol_w);
+      else
+        tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, (c.kb0 + c.i) * GEMM_BK, c.n0 + h * GEMM_BM, pol_w);
+  };
+  auto load_b = [&](const Cursor& c, int it) {
+    const int s = it % STAGES;
+    tma_load_2d_hint(smem_base + s * p.stage_bytes + a_bytes, &tm_x, smem_u32(&bars[s]), (c.kb0 + c.i) * GEMM_BK,
+                     c.r0, pol_x);
+  };
+  head = cur;
+  int pre = 0;
+
+  pdl_launch();   // the next kernel in the stream may start its own prologue
   if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tm_w);
+    tma_prefetch_desc(&tm_x);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&bars[s]), 1);
       mbar_init(smem_u32(&bars[STAGES + s]), 1);
@@ -332,82 +385,29 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
+    Cursor c = cur;
+    while (p.w_static && pre < STAGES && settle(c)) {   // all stages are free at the start: no wait needed
+      load_a(c, pre);
+      ++pre;
+      ++c.i;
+    }
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_slot), p.tmem_cols);
     tmem_relinquish();
-  }
-  if (warp == 0 && lane == 0) {
-    tma_prefetch_desc(&tm_w);
-    tma_prefetch_desc(&tm_x);
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // unit u -> (weight tile, row tile, split); consecutive units differ in the split first
-  auto decode = [&](int u, int& n0, int& r0, int& split, int& kb0, int& n_kb) {
-    split = u % p.splits;
-    const int t = u / p.splits;
-    r0 = (t % p.r_tiles) * p.br;
-    n0 = (t / p.r_tiles) * tile_rows;
-    kb0 = split * p.kb_per_split;
-    n_kb = max(0, min(p.kb_total, kb0 + p.kb_per_split) - kb0);
-  };
-
   const unsigned long long t_enter = (trace_on() && threadIdx.x == 64) ? global_timer_ns() : 0ull;
-  pdl_launch();   // the next kernel in the stream may start its own prologue
 
   if (warp == 0) {
     // ------------------------------------------------------- TMA producer
     if (lane == 0) {
-      const uint64_t pol_w = l2_policy_evict_first();   // weights are streamed once per step
-      const uint64_t pol_x = l2_policy_evict_last();    // the few activation rows are re-read by every CTA
-      // The weights never change, so the ring is first filled with weight
-      // tiles alone; only the activation rows have to wait for the kernel
-      // that produces them.
-      struct Cursor {
-        int u, i, n0, r0, split, kb0, n_kb;
-      } cur, head;
-      cur.u = blockIdx.x;
-      cur.i = 0;
-      auto settle = [&](Cursor& c) {   // move to the next k-block that exists (or past the end)
-        while (c.u < p.units) {
-          decode(c.u, c.n0, c.r0, c.split, c.kb0, c.n_kb);
-          if (c.i < c.n_kb) return true;
-          c.u += gridDim.x;
-          c.i = 0;
-        }
-        return false;
-      };
-      auto load_a = [&](const Cursor& c, int it) {
-        const int s = it % STAGES;
-        const uint32_t full = smem_u32(&bars[s]);
-        mbar_expect_tx(full, static_cast<uint32_t>(p.stage_bytes));
-        const uint32_t a_dst = smem_base + s * p.stage_bytes;
-        for (int h = 0; h < p.halves; ++h)
-          if (p.w_blocked)      // block (row block, k-block) of a blocked copy: rows block * 128 .. + 127 of its map
-            tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, 0,
-                             (c.n0 + h * GEMM_BM) * p.kb_total + (c.kb0 + c.i) * GEMM_BM, pol_w);
-          else
-            tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, (c.kb0 + c.i) * GEMM_BK, c.n0 + h * GEMM_BM, pol_w);
-      };
-      auto load_b = [&](const Cursor& c, int it) {
-        const int s = it % STAGES;
-        tma_load_2d_hint(smem_base + s * p.stage_bytes + a_bytes, &tm_x, smem_u32(&bars[s]), (c.kb0 + c.i) * GEMM_BK,
-                         c.r0, pol_x);
-      };
-      head = cur;
-      int pre = 0;
-      Cursor c = cur;
-      while (p.w_static && pre < STAGES && settle(c)) {   // all stages are free at the start: no wait needed
-        load_a(c, pre);
-        ++pre;
-        ++c.i;
-      }
       pdl_wait();
-      c = head;
+      Cursor c = head;
       for (int it = 0; it < pre; ++it) {
         settle(c);
         load_b(c, it);
