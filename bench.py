@@ -740,6 +740,48 @@ def run_layer_sweep(args):
                 torch.cuda.empty_cache()
 
 
+def run_stream_sweep(args):
+    """The memory side of a weight-streaming launch alone (`dkv_op_stream_probe`: bulk copies into a ring
+    of shared-memory stages, no arithmetic): 201 MB (the gate/up matrix of an LLaDA-shaped layer) of
+    unique bytes per launch, with and without bytes that every CTA re-reads from L2, over the number of
+    CTAs and the ring depth.  One JSON line per point: time per launch (eight launches back to back
+    between two events, each on another L2-cold window) and TB/s."""
+    import torch
+    from paper_2505_15781_b200 import binding as B
+    torch.cuda.set_device(0)
+    total = 201 << 20
+    big = torch.ones(1 << 30, dtype=torch.uint8, device="cuda")          # four disjoint 256 MB windows: cold in L2
+    small = torch.ones(1179648, dtype=torch.uint8, device="cuda")        # 144 rows x 4096 x 2 bytes
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for ctas in (74, 96, 128, 148):
+        for b_kb in (0, 9, 18):
+            for stages in (3, 4, 6):
+                if (32 + b_kb) * stages > 216:
+                    continue
+                def launch(r):
+                    win = big[(r % 4) * (256 << 20):(r % 4) * (256 << 20) + total]
+                    B.dkv_op_stream_probe(win, small if b_kb else None, ctas, 32 << 10, b_kb << 10, stages, status)
+                ts = []
+                for rep in range(4):      # rep 0 is the warm-up; 8 launches back to back between two events
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for r in range(8):
+                        launch(r)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if rep:
+                        ts.append(e0.elapsed_time(e1) * 1e-3 / 8)
+                t = sum(ts) / len(ts)
+                moved = total // ctas // (32 << 10) * (32 << 10) * ctas
+                reread = total // ctas // (32 << 10) * (b_kb << 10) * ctas
+                print(json.dumps({"sweep": "stream", "ctas": ctas, "streamed_kb_per_stage": 32, "reread_kb_per_stage": b_kb,
+                                  "stages": stages, "launch_us": round(t * 1e6, 1), "best_us": round(min(ts) * 1e6, 1),
+                                  "streamed_TBps": round(moved / t / 1e12, 2),
+                                  "streamed_plus_reread_TBps": round((moved + reread) / t / 1e12, 2),
+                                  "status": int(status.item())}), flush=True)
+
+
 def run_attention_sweep(args):
     """The attention kernel alone (`dkv_op_attention`, fp16, head_dim 128) over (rows, slots, batch,
     query heads, KV heads) cases: time, TFLOP/s (4*rows*slots*d_q), GB/s of slots + queries + outputs."""
@@ -779,7 +821,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b_decode", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", default="", choices=["", "batch", "layer", "attention", "order", "length"])
+    ap.add_argument("--sweep", default="", choices=["", "batch", "layer", "attention", "order", "length", "stream"])
     ap.add_argument("--sweep-gens", default="128,256,512,1024")
     ap.add_argument("--sweep-prompts", default="0,128,512,2048")
     ap.add_argument("--attn-cases", default="254x512x1x32x32,512x512x1x32x32,1024x1024x8x32x32,4096x4096x1x32x32,"
@@ -793,6 +835,9 @@ def main():
     if args.sweep == "batch":
         args.sweep_batches = args.sweep_batches or "1,2,4,8,16,32,64"
         run_batch_sweep(args)
+        return
+    if args.sweep == "stream":
+        run_stream_sweep(args)
         return
     if args.sweep == "attention":
         args.steps = min(args.steps, 10)

@@ -393,6 +393,23 @@ size_t dkv_static_scratch_bytes(void);
 int dkv_op_gemm_static(const void* x, const void* w, float* out, int rows, int n, int k, int dtype, int splits,
                        void* stream);
 
+/* Measurement aid (no counterpart in the paper): the memory side of a
+ * weight-streaming projection launch without its arithmetic.  `ctas` thread
+ * blocks (one per SM) each stream their own slice of `streamed` (unique
+ * bytes, meant to come from HBM: make the buffer larger than L2) and, per
+ * chunk, reread_chunk_bytes of the small buffer `reread` that every block
+ * re-reads (L2 hits, like the activation rows of a projection; 0 = none),
+ * through a ring of `stages` shared-memory stages filled by bulk copies; a
+ * stage is freed the moment it is full.  Every block moves
+ * floor(streamed_bytes / ctas / chunk_bytes) chunks.  The launch's duration
+ * (time it with events on `stream`) is the ceiling of that access pattern.
+ * Both buffers 16-byte aligned device memory, the chunk sizes multiples of 16,
+ * stages * (chunk_bytes + reread_chunk_bytes) at most about 226 KB.  `status`
+ * (device int32, may be NULL): bit 3 is set if a bounded wait ran out.
+ * Errors: INVALID_ARG, SHAPE, NOMEM (shared memory), CUDA. */
+int dkv_op_stream_probe(const void* streamed, long long streamed_bytes, const void* reread, long long reread_bytes,
+                        int ctas, int chunk_bytes, int reread_chunk_bytes, int stages, int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ EXPORTS = [
     "dkv_get_stats", "dkv_get_provenance", "dkv_get_index_maps", "dkv_status", "dkv_cache_slots",
     "dkv_profile_enable", "dkv_profile_read", "dkv_gemm_workspace_bytes", "dkv_op_gemm", "dkv_op_attention",
     "dkv_static_scratch_bytes", "dkv_op_gemm_static", "dkv_trace_set", "dkv_debug_tail_wait",
-    "dkv_cache_state_bytes", "dkv_cache_export", "dkv_cache_import",
+    "dkv_cache_state_bytes", "dkv_cache_export", "dkv_cache_import", "dkv_op_stream_probe",
 ]
 
 
@@ -121,6 +121,7 @@ def load():
     lib.dkv_static_scratch_bytes.restype = sz
     lib.dkv_static_scratch_bytes.argtypes = []
     lib.dkv_op_gemm_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+    lib.dkv_op_stream_probe.argtypes = [vp, C.c_longlong, vp, C.c_longlong, i32, i32, i32, i32, vp, vp]
     for name in EXPORTS:
         if name not in ("dkv_strerror", "dkv_model_bytes", "dkv_cache_bytes", "dkv_gemm_workspace_bytes",
                         "dkv_static_scratch_bytes", "dkv_cache_state_bytes"):
@@ -332,6 +333,14 @@ def dkv_profile_read(cache: Cache) -> List[dict]:
     _check("dkv_profile_read", load().dkv_profile_read(cache.handle, arr, C.byref(n)))
     return [dict(name=arr[i].name.decode(), launches=arr[i].launches, ms=arr[i].ms, bytes=arr[i].bytes,
                  flops=arr[i].flops) for i in range(n.value)]
+
+
+def dkv_op_stream_probe(streamed, reread, ctas: int, chunk_bytes: int, reread_chunk_bytes: int, stages: int,
+                        status=None, stream=None):
+    """streamed / reread: CUDA uint8 tensors (reread may be None when reread_chunk_bytes is 0)."""
+    _check("dkv_op_stream_probe", load().dkv_op_stream_probe(
+        _ptr(streamed), streamed.numel(), _ptr(reread), reread.numel() if reread is not None else 0, ctas,
+        chunk_bytes, reread_chunk_bytes, stages, _ptr(status), _stream(stream)))
 
 
 def dkv_gemm_workspace_bytes(rows: int, n: int) -> int:

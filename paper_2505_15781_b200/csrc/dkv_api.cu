@@ -22,6 +22,7 @@
 #include "gemm_tc2.cuh"
 #include "attn_tc.cuh"
 #include "index_kernels.cuh"
+#include "stream_probe.cuh"
 #include "ptx.cuh"
 #include "row_kernels.cuh"
 
@@ -1916,6 +1917,35 @@ int dkv_op_gemm_static(const void* x, const void* w, float* out, int rows, int n
   const long long elems = static_cast<long long>(rows) * n;
   launch_k(k_reduce_partials, static_cast<int>(std::min<long long>(4 * NUM_SMS, (elems + 255) / 256)), 256, 0, st,
            static_cast<const float*>(scratch), s, stride, rows, static_cast<const int*>(nullptr), n, out);
+  return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
+}
+
+int dkv_op_stream_probe(const void* streamed, long long streamed_bytes, const void* reread, long long reread_bytes,
+                        int ctas, int chunk_bytes, int reread_chunk_bytes, int stages, int32_t* status, void* stream) {
+  if (!streamed) return DKV_E_INVALID_ARG;
+  if (ctas < 1 || ctas > 1024 || stages < 1 || stages > 32) return DKV_E_SHAPE;
+  if (chunk_bytes < 16 || chunk_bytes % 16 || reread_chunk_bytes < 0 || reread_chunk_bytes % 16) return DKV_E_SHAPE;
+  if (reread_chunk_bytes > 0 && (!reread || reread_bytes < reread_chunk_bytes)) return DKV_E_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(streamed) % 16 || reinterpret_cast<uintptr_t>(reread) % 16) return DKV_E_INVALID_ARG;
+  const size_t smem = static_cast<size_t>(stages) * (chunk_bytes + reread_chunk_bytes) + 2 * stages * 8 + 16;
+  if (smem > 227 * 1024) return DKV_E_NOMEM;
+  StreamProbeParams p;
+  p.a = static_cast<const uint8_t*>(streamed);
+  p.b = static_cast<const uint8_t*>(reread);
+  p.n_chunks = static_cast<int>(std::min<long long>(streamed_bytes / ctas / chunk_bytes, 1 << 30));
+  if (p.n_chunks < 1) return DKV_E_SHAPE;
+  p.a_per_cta = static_cast<long long>(p.n_chunks) * chunk_bytes;
+  p.a_chunk = chunk_bytes;
+  p.b_chunk = reread_chunk_bytes;
+  p.b_span = reread_chunk_bytes > 0 ? reread_bytes / reread_chunk_bytes * reread_chunk_bytes : 0;
+  p.stages = stages;
+  p.wait_cycles = GEMM_WAIT_CYCLES;
+  p.status = status;
+  static PerDeviceOnce attr_once;
+  if (attr_once.need() &&
+      cudaFuncSetAttribute(k_stream_probe, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    return DKV_E_CUDA;
+  k_stream_probe<<<ctas, 64, smem, static_cast<cudaStream_t>(stream)>>>(p);
   return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;
 }
 

@@ -150,3 +150,22 @@ def test_generator_is_identical_on_device():
     np.testing.assert_array_equal(a, synth.hash_u16_numpy(11, 200000, k1, k2))
     w = synth.normal_tensor(0, 1, "wd", (96, 200), 0.02, "bfloat16", "cuda")
     assert torch.equal(w.cpu(), synth.normal_tensor(0, 1, "wd", (96, 200), 0.02, "bfloat16", "cpu"))
+
+
+def test_stream_probe_runs_to_completion_and_checks_its_arguments():
+    """The measurement kernel (a ring of bulk copies without arithmetic) moves every chunk, reports no
+    wait that ran out, and the entry point refuses sizes the copy engine cannot take."""
+    lib = B.load()
+    streamed = torch.ones(64 << 20, dtype=torch.uint8, device="cuda")
+    reread = torch.ones(1 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for ctas, chunk, rechunk, stages in ((148, 32 << 10, 18 << 10, 4), (3, 16, 0, 1), (96, 32 << 10, 9 << 10, 5)):
+        B.dkv_op_stream_probe(streamed, reread if rechunk else None, ctas, chunk, rechunk, stages, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    args = (streamed.data_ptr(), streamed.numel(), reread.data_ptr(), reread.numel())
+    assert lib.dkv_op_stream_probe(*args, 148, 24, 0, 4, None, None) == -2               # chunk not a multiple of 16
+    assert lib.dkv_op_stream_probe(*args, 148, 64 << 10, 0, 4, None, None) == -4         # ring larger than shared memory
+    assert lib.dkv_op_stream_probe(*args, 0, 1024, 0, 4, None, None) == -2
+    assert lib.dkv_op_stream_probe(None, 1 << 20, None, 0, 8, 1024, 0, 4, None, None) == -1
+    assert lib.dkv_op_stream_probe(args[0], args[1], None, 0, 8, 1024, 512, 4, None, None) == -1   # re-read buffer missing
