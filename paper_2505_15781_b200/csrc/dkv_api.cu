@@ -383,7 +383,7 @@ struct dkv_cache {
   dkv_policy policy;
   Arena ar;
   CUtensorMap xmaps[XB_COUNT][N_BOX];
-  CUtensorMap xmaps_half[N_BOX];   // the normalised rows (XB_XN) in boxes of half the rows, for the CTA-pair GEMM
+  CUtensorMap xmaps_half[XB_COUNT][N_BOX];   // the same operands in boxes of half the rows, for the CTA-pair GEMM
   AttnMaps attn_maps;            // tcgen05 attention (head_dim 128, 16-bit modes): all seq_len slots attended
   AttnMaps attn_maps_prompt;     // the same buffers with the slot extent cut at the prompt (isolated prefill pass)
   bool attn_tc;
@@ -526,6 +526,44 @@ void choose_multi_tile(int n, int k, int r_bound, long long part_rows, int* tile
   }
 }
 
+// The same estimate for a launch on CTA pairs (k_gemm_tc2): a unit is 512 weight rows x br rows on two
+// SMs, each CTA takes in 32 KB of weights and br / 2 rows per k-block, and the units run in waves of
+// NUM_SMS / 2 pairs.  `one_wave`: only plans whose units are all resident at once (fused row tails).
+double est_clocks_pairs(int n, int k, int r_bound, int t, int s) {
+  const int per = ceil_div(r_bound, t);
+  const int br = 16 * ceil_div(per, 16);
+  const int kb_total = ceil_div(k, GEMM_BK);
+  const double kbu = std::ceil(kb_total / static_cast<double>(s));
+  const double cyc_kb = std::max(4.0 * br, (2.0 * GEMM_A_BYTES + 64.0 * br) / 52.0);
+  const double unit = kbu * cyc_kb + br * 1024.0 / 64.0;
+  const double units = static_cast<double>(ceil_div(n, 512)) * t * s;
+  const double waves = std::ceil(units / (NUM_SMS / 2));
+  const double partials = s > 1 ? 4.0 * s * r_bound * static_cast<double>(n) / (4.0e12 / 1.85e9) : 0.0;
+  return waves * unit + partials;
+}
+double choose_pairs(int n, int k, int r_bound, long long part_rows, bool one_wave, int* tiles_out, int* splits_out) {
+  const int kb_total = ceil_div(k, GEMM_BK);
+  int s_max = std::min(8, std::max(1, kb_total / 4));
+  s_max = static_cast<int>(std::min<long long>(s_max, std::max<long long>(1, part_rows / std::max(1, r_bound))));
+  const int t_min = ceil_div(r_bound, 256);
+  double best = 1e300;
+  *tiles_out = 0;
+  *splits_out = 0;
+  for (int t = t_min; t <= t_min + 2; ++t) {
+    for (int s = 1; s <= s_max; ++s) {
+      if (s > 1 && (s - 1) * ceil_div(kb_total, s) >= kb_total) continue;
+      if (one_wave && ceil_div(n, 512) * t * s > NUM_SMS / 2) continue;
+      const double c = est_clocks_pairs(n, k, r_bound, t, s);
+      if (c < best * 0.97) {
+        best = c;
+        *tiles_out = t;
+        *splits_out = s;
+      }
+    }
+  }
+  return best;
+}
+
 int env_int(const char* name, int dflt) {
   const char* s = getenv(name);
   return s ? atoi(s) : dflt;
@@ -609,6 +647,27 @@ struct GemmOpts {
   FusedTail tail;                            // applied only when the launch is one wave (see *fused_out)
 };
 
+void set_tail(GemmTcParams& p, const FusedTail& t) {
+  p.fuse_mode = t.mode;
+  p.tile_cnt = t.tile_cnt;
+  p.tail_wait_cycles = t.wait_cycles;
+  p.tail_extra = t.extra;
+  p.h = t.h;
+  p.gain = t.gain;
+  p.xn_out = t.xn_out;
+  p.ssq_out = t.ssq_out;
+  p.ssq_ld = t.ssq_ld;
+  p.act_idx = t.act_idx;
+  p.rope_tab = t.rope_tab;
+  p.seq_len = t.seq_len;
+  p.n_q_heads = t.n_q_heads;
+  p.n_kv_heads = t.n_kv_heads;
+  p.head_dim = t.head_dim;
+  p.q_out = t.q_out;
+  p.k_slots = t.k_slots;
+  p.v_slots = t.v_slots;
+}
+
 // out (fp32 partials) [splits][r_bound * n]; returns splits and stride through the pointers.  When a
 // fused tail is asked for and every unit gets a CTA of its own (units <= SMs, so that the CTAs of a
 // tile can wait for each other), the kernel runs it and *fused_out is true; otherwise the partials
@@ -665,6 +724,12 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
     p.r_tiles = ceil_div(r_bound, br);
     p.units = ceil_div(n, GEMM2_TILE_ROWS) * p.r_tiles * splits;
     const int grid = 2 * std::min(p.units, NUM_SMS / 2);
+    // fused row tails: each CTA of a pair is a 256-column tile of its own; all units resident at once
+    if (o.tail.mode != FUSE_NONE && !o.swiglu_out && p.units <= NUM_SMS / 2 &&
+        2 * ceil_div(n, GEMM2_TILE_ROWS) * p.r_tiles <= MAX_TILE_COUNTERS) {
+      set_tail(p, o.tail);
+      if (fused_out) *fused_out = true;
+    }
     launch_k(k_gemm_tc2, grid, GEMM_THREADS, plan.smem_bytes, st, tw, o.xmaps_half[bi], p);
     *splits_out = splits;
     *stride_out = p.split_stride;
@@ -713,25 +778,7 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
   }
   // the CTAs of a tile wait for each other in the fused tail: every unit needs a resident CTA of its own
   if (o.tail.mode != FUSE_NONE && p.units <= sms && p.units <= MAX_TILE_COUNTERS) {
-    const FusedTail& t = o.tail;
-    p.fuse_mode = t.mode;
-    p.tile_cnt = t.tile_cnt;
-    p.tail_wait_cycles = t.wait_cycles;
-    p.tail_extra = t.extra;
-    p.h = t.h;
-    p.gain = t.gain;
-    p.xn_out = t.xn_out;
-    p.ssq_out = t.ssq_out;
-    p.ssq_ld = t.ssq_ld;
-    p.act_idx = t.act_idx;
-    p.rope_tab = t.rope_tab;
-    p.seq_len = t.seq_len;
-    p.n_q_heads = t.n_q_heads;
-    p.n_kv_heads = t.n_kv_heads;
-    p.head_dim = t.head_dim;
-    p.q_out = t.q_out;
-    p.k_slots = t.k_slots;
-    p.v_slots = t.v_slots;
+    set_tail(p, o.tail);
     if (fused_out) *fused_out = true;
   }
   launch_k(k_gemm_tc, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps[bi], p);
@@ -886,6 +933,22 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     scale_from(1);
   };
 
+  // More than one row tile (the full steps): the launch is bound by the operand bytes an SM takes in
+  // and by the power cap, and a CTA pair (each CTA stages half of the row tile) takes in a quarter
+  // less per flop: QKV 57 -> 55 us, O 42 -> 40, down 65 -> 62 at 512 LLaDA-shaped rows.  Row tiles and
+  // K splits from the estimate for pairs; `one_wave`: prefer a plan that leaves every unit resident,
+  // so that the residual tail can be fused.
+  auto pair_plan = [&](GemmOpts& o, XBuf xb, int n, int k, bool one_wave) {
+    if (!bf16 || R <= 256 || !m->gu_pair) return;
+    int t = 0, sp = 0;
+    choose_pairs(n, k, R, dm.part_rows, one_wave, &t, &sp);
+    if (t == 0 && one_wave) choose_pairs(n, k, R, dm.part_rows, false, &t, &sp);
+    if (t == 0) return;
+    o.xmaps_half = c->xmaps_half[xb];
+    o.row_tiles = t;
+    o.forced_splits = sp;
+  };
+
   {
     Launch l(c, st, PC_EMBED, R * d * (es + 4.0 + es), 0);
     launch_k((k_embed_norm<TW, T>), R, 256, 0, st, static_cast<const TW*>(m->embed), tokens, a.act_idx, r_dev,
@@ -924,8 +987,10 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     int splits;
     long long stride;
     bool fused;
+    GemmOpts oq = qkv_opts(l);
+    pair_plan(oq, XB_XN, nqkv, d, false);
     rc = gemm(PC_GEMM_QKV, lw.wqkv, lm ? &lm->wqkv : nullptr, XB_XN, a.xn, nqkv, d, R, r_dev, a.part, &splits, &stride,
-              qkv_opts(l), &fused);
+              oq, &fused);
     if (rc) return rc;
     if (!fused) {
       Launch lk(c, st, PC_QKV_POST, R * (nqkv * 4.0 * splits + nqkv * es), 0);
@@ -951,8 +1016,9 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       if (rc) return rc;
     }
     const float* next_gain = (l + 1 < md.n_layers) ? m->layers[l + 1].attn_norm : m->final_norm;
-    rc = gemm(PC_GEMM_O, lw.wo, lm ? &lm->wo : nullptr, XB_AO, a.ao, d, dq, R, r_dev, a.part, &splits, &stride,
-              resid_opts(lw.ffn_norm), &fused);
+    GemmOpts oo = resid_opts(lw.ffn_norm);
+    pair_plan(oo, XB_AO, d, dq, oo.tail.mode != FUSE_NONE);
+    rc = gemm(PC_GEMM_O, lw.wo, lm ? &lm->wo : nullptr, XB_AO, a.ao, d, dq, R, r_dev, a.part, &splits, &stride, oo, &fused);
     if (rc) return rc;
     resid_after(fused, splits, stride, lw.ffn_norm);
     // The SwiGLU epilogue needs the whole K range in one unit (no split-K).  With one row tile that
@@ -980,7 +1046,7 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       o.scale = sc;
       o.swiglu_out = a.ub;
       o.ld_u = f;
-      o.xmaps_half = m->gu_pair ? c->xmaps_half : nullptr;
+      o.xmaps_half = m->gu_pair ? c->xmaps_half[XB_XN] : nullptr;
       o.row_tiles = R > 256 ? gu_rt : 0;
       o.w_blocked = m->w_blocked;
       rc = gemm_tc(lm->wgu, c->xmaps[XB_XN], 2 * f, d, R, r_dev, a.part, dm.part_rows, a.status, x_bf16, st, &splits,
@@ -996,8 +1062,9 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
       launch_k((k_swiglu<T>), grid, 256, 0, st, a.part, splits, stride, r_dev, f, bf16 ? m->gu_blk : 0,
                static_cast<T*>(a.ub));
     }
-    rc = gemm(PC_GEMM_DOWN, lw.wd, lm ? &lm->wd : nullptr, XB_U, a.ub, d, f, R, r_dev, a.part, &splits, &stride,
-              resid_opts(next_gain), &fused);
+    GemmOpts od = resid_opts(next_gain);
+    pair_plan(od, XB_U, d, f, od.tail.mode != FUSE_NONE);
+    rc = gemm(PC_GEMM_DOWN, lw.wd, lm ? &lm->wd : nullptr, XB_U, a.ub, d, f, R, r_dev, a.part, &splits, &stride, od, &fused);
     if (rc) return rc;
     resid_after(fused, splits, stride, next_gain);
   }
@@ -1366,9 +1433,11 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
     for (int i = 0; i < N_BOX && !rc; ++i) {
       const bool h = md.act_dtype == DKV_F16;
       rc = make_tmap(&c->xmaps[XB_XN][i], a.xn, c->dims.r_cap, md.d_model, box_rows(i), h);
-      if (!rc) rc = make_tmap(&c->xmaps_half[i], a.xn, c->dims.r_cap, md.d_model, box_rows(i) / 2, h);
+      if (!rc) rc = make_tmap(&c->xmaps_half[XB_XN][i], a.xn, c->dims.r_cap, md.d_model, box_rows(i) / 2, h);
       if (!rc) rc = make_tmap(&c->xmaps[XB_AO][i], a.ao, c->dims.r_cap, m->d_q, box_rows(i), h);
+      if (!rc) rc = make_tmap(&c->xmaps_half[XB_AO][i], a.ao, c->dims.r_cap, m->d_q, box_rows(i) / 2, h);
       if (!rc) rc = make_tmap(&c->xmaps[XB_U][i], a.ub, c->dims.r_cap, md.d_ffn, box_rows(i), h);
+      if (!rc) rc = make_tmap(&c->xmaps_half[XB_U][i], a.ub, c->dims.r_cap, md.d_ffn, box_rows(i) / 2, h);
       if (!rc) rc = make_tmap(&c->xmaps[XB_XH][i], a.xh, c->dims.h_cap, md.d_model, box_rows(i), h);
     }
     c->attn_tc = false;

@@ -244,7 +244,7 @@ __device__ __forceinline__ void fused_rows_resid(const GemmTcParams& p, int n0, 
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      if (lane == 0 && rb + rr < row_hi) p.ssq_out[tile_n * p.ssq_ld + rb + rr] = ss;
+      if (lane == 0 && rb + rr < row_hi && n0 < p.n) p.ssq_out[tile_n * p.ssq_ld + rb + rr] = ss;   // (a pair's second CTA may own no column)
     }
   }
 }
@@ -299,6 +299,39 @@ __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, in
       *reinterpret_cast<uint2*>(dst + i0 + half) = pack4_16(x2.x, x2.y, x2.z, x2.w, p.x_bf16);
     }
   }
+}
+
+// Cross-CTA hand-over of the fused row epilogues, run by the 256 epilogue threads of a CTA after its
+// partial sums of the unit are in scratch: the CTA counts itself on the tile's counter and waits
+// (bounded) until all K splits of the tile are there; then it finishes its own slice of the tile's
+// rows.  `tile` indexes the counters; the tile's columns are [n0, n0 + tile_rows).  The last CTA to
+// get past the wait resets the counter.  Returns false when a wait ran out (the abort flag is set).
+__device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int split, int n0, int tile_rows, int r0,
+                                           int r_valid, volatile int* abort_flag, int et, int ewarp, int lane) {
+  unsigned int* cnt = p.tile_cnt + tile;
+  __threadfence();
+  named_bar_sync(2, 256);
+  bool fail = false;
+  if (et == 0) {
+    atomicAdd(cnt, 1u);
+    const long long t0 = clock64();
+    while (ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits + p.tail_extra)) {
+      if (*abort_flag || clock64() - t0 > p.tail_wait_cycles) {
+        fail = true;
+        *abort_flag = 1;
+        break;
+      }
+    }
+    if (!fail && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;   // everyone has passed: reset
+    __threadfence();
+  }
+  if (bar_red_or(2, 256, fail)) return false;
+  const int n_rows = max(0, min(p.br, r_valid - r0));
+  const int per = (n_rows + p.splits - 1) / p.splits;
+  const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
+  if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, ewarp, lane);
+  else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, ewarp, lane);
+  return true;
 }
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -631,37 +664,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
 
-      if (p.fuse_mode != FUSE_NONE) {
-        // Cross-CTA hand-over: this CTA's partial sums are in scratch; count it on the tile's counter
-        // and wait until all K splits of the tile are there.  Then every CTA of the tile finishes its
-        // own slice of the tile's rows.  The last CTA to get past the wait resets the counter.
-        const int tile = u / p.splits;
-        unsigned int* cnt = p.tile_cnt + tile;
-        __threadfence();
-        named_bar_sync(2, 256);
-        bool fail = false;
-        if (et == 0) {
-          atomicAdd(cnt, 1u);
-          const long long t0 = clock64();
-          while (ld_acquire_gpu(cnt) < static_cast<unsigned int>(p.splits + p.tail_extra)) {
-            if (*abort_flag || clock64() - t0 > p.tail_wait_cycles) {
-              fail = true;
-              *abort_flag = 1;
-              break;
-            }
-          }
-          if (!fail && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;   // everyone has passed: reset
-          __threadfence();
-        }
-        if (bar_red_or(2, 256, fail)) {
-          ok = false;
-          break;
-        }
-        const int n_rows = max(0, min(p.br, r_valid - r0));
-        const int per = (n_rows + p.splits - 1) / p.splits;
-        const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
-        if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
-        else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, warp - 2, lane);
+      if (p.fuse_mode != FUSE_NONE &&
+          !fused_tail(p, u / p.splits, split, n0, tile_rows, r0, r_valid, abort_flag, et, warp - 2, lane)) {
+        ok = false;
+        break;
       }
     }
     if (p.head_mode && ok && lane < 16) {

@@ -5,11 +5,14 @@
 // memory).  Per 32 KB of weights a CTA therefore holds br * 64 bytes of rows
 // instead of br * 128: the ring is deeper at the same shared memory and the
 // L2 -> SM traffic of the rows halves, which is what bounds the one-CTA kernel
-// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).  The kernel serves ONE
-// launch: the unsplit gate/up projection with the SwiGLU epilogue (the split-K launches gain nothing from
-// pairs).  Which 128 rows a CTA stages for MMA h is a matter of its TMA coordinate only: rank r takes rows
-// [r*256 + h*128, +128) of the weight copy grouped [128 gate | 128 up] per 256 rows, so that each CTA
-// holds the gate rows (MMA 0) and the up rows (MMA 1) of the same 128 features.
+// above ~128 rows.  A pair's tile is 512 weight rows (two MMAs side by side).  Which 128 rows a CTA
+// stages for MMA h is a matter of its TMA coordinate only: rank r takes rows [r*256 + h*128, +128), so
+// a CTA always owns 256 consecutive rows of the weight matrix.  Two uses: the unsplit gate/up
+// projection with the SwiGLU epilogue (the weight copy is grouped [128 gate | 128 up] per 256 rows,
+// so that each CTA holds the gate rows (MMA 0) and the up rows (MMA 1) of the same 128 features),
+// and the QKV / O / down projections of steps with more than one row tile, with plain fp32 partial
+// sums and, for O and down, the fused residual tail of k_gemm_tc (each CTA of a pair then counts as
+// a 256-column weight tile of its own).  The split-K launches of the cached steps gain nothing from pairs.
 //
 // Roles per CTA (320 threads): warp 0 = TMA producer of its own half of the
 // operands, completion counted on the LEADER's barrier (cta_group::2 loads);
@@ -291,7 +294,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
       tc_fence_after();
       const int row_in_tile = static_cast<int>(rank) * GEMM_BM + q * 32 + lane;
       const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(buf * 2 * p.col_stride);
-      {
+      if (p.swiglu_out) {
         // the gate/up copy is grouped [128 gate rows | 128 up rows] per 256 rows and this CTA staged the
         // gate rows (MMA 0) and the up rows (MMA 1) of features (n0 / 2) + rank * 128 + [0, 128)
         const int jf = (n0 >> 1) + row_in_tile;
@@ -332,11 +335,51 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
             }
           }
         }
+      } else {
+        // plain partial sums: this CTA holds weight rows n0 + rank * 256 + h * 128 + [0, 128) in MMA h,
+        // i.e. 256 consecutive output columns, like one tile of the one-CTA kernel
+        float* out = p.out + static_cast<long long>(split) * p.split_stride;
+        for (int h = 0; h < 2; ++h) {
+          const int n = n0 + static_cast<int>(rank) * 256 + h * GEMM_BM + q * 32 + lane;
+          const uint32_t t_addr = t_lane + static_cast<uint32_t>(h * p.col_stride);
+          for (int c = cs * 16; c < p.br; c += 32) {
+            if (r0 + c >= r_valid) break;
+            uint32_t v[16];
+            if (n_kb > 0) {
+              tmem_ld_x16(t_addr + c, v);
+              tmem_ld_wait();
+#pragma unroll
+              for (int jj = 0; jj < 16; ++jj) v[jj] = __float_as_uint(__uint_as_float(v[jj]) * s_rs[c + jj]);
+            } else {
+#pragma unroll
+              for (int jj = 0; jj < 16; ++jj) v[jj] = 0u;
+            }
+            if (n < p.n) {
+              float* dst = out + static_cast<long long>(r0 + c) * p.ldo + n;
+              if (r0 + c + 16 <= r_valid) {
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) dst[static_cast<long long>(jj) * p.ldo] = __uint_as_float(v[jj]);
+              } else {
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj)
+                  if (r0 + c + jj < r_valid) dst[static_cast<long long>(jj) * p.ldo] = __uint_as_float(v[jj]);
+              }
+            }
+          }
+        }
       }
       // this warp is done reading the buffer: tell the leader's MMA thread
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&acc_empty[buf]), 0));
+
+      // fused row epilogue across the K splits: each CTA of the pair is one 256-column tile of its own
+      if (p.fuse_mode != FUSE_NONE &&
+          !fused_tail(p, (u / p.splits) * 2 + static_cast<int>(rank), split, n0 + static_cast<int>(rank) * 256, 256, r0,
+                      r_valid, abort_flag, et, warp - 2, lane)) {
+        ok = false;
+        break;
+      }
     }
   }
 
