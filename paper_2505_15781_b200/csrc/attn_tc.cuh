@@ -406,23 +406,29 @@ k_attn_tc(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const float inv = 1.f / l_row;
         uint8_t* orow = static_cast<uint8_t*>(p.o) +
                         ((static_cast<long long>(p.row_off[b] + q0 + qi) * p.n_q_heads + hk * p.group + g) * ATC_DH) * 2;
+        // the thread's columns in groups of 64: all four tensor-memory loads of a group are in flight
+        // before the one wait (one round trip instead of four)
 #pragma unroll
-        for (int c = wg * O_COLS; c < wg * O_COLS + O_COLS; c += 16) {
-          uint32_t v[16];
-          tmem_ld_x16(tO + lane_addr + c, v);
+        for (int c0 = wg * O_COLS; c0 < wg * O_COLS + O_COLS; c0 += 64) {
+          uint32_t v[4][16];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) tmem_ld_x16(tO + lane_addr + c0 + g * 16, v[g]);
           tmem_ld_wait();
           if (valid) {
-            uint4 w0, w1;
-            w0.x = pack16(__uint_as_float(v[0]) * inv, __uint_as_float(v[1]) * inv, p.bf16);
-            w0.y = pack16(__uint_as_float(v[2]) * inv, __uint_as_float(v[3]) * inv, p.bf16);
-            w0.z = pack16(__uint_as_float(v[4]) * inv, __uint_as_float(v[5]) * inv, p.bf16);
-            w0.w = pack16(__uint_as_float(v[6]) * inv, __uint_as_float(v[7]) * inv, p.bf16);
-            w1.x = pack16(__uint_as_float(v[8]) * inv, __uint_as_float(v[9]) * inv, p.bf16);
-            w1.y = pack16(__uint_as_float(v[10]) * inv, __uint_as_float(v[11]) * inv, p.bf16);
-            w1.z = pack16(__uint_as_float(v[12]) * inv, __uint_as_float(v[13]) * inv, p.bf16);
-            w1.w = pack16(__uint_as_float(v[14]) * inv, __uint_as_float(v[15]) * inv, p.bf16);
-            *reinterpret_cast<uint4*>(orow + c * 2) = w0;
-            *reinterpret_cast<uint4*>(orow + c * 2 + 16) = w1;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 w0, w1;
+              w0.x = pack16(__uint_as_float(v[g][0]) * inv, __uint_as_float(v[g][1]) * inv, p.bf16);
+              w0.y = pack16(__uint_as_float(v[g][2]) * inv, __uint_as_float(v[g][3]) * inv, p.bf16);
+              w0.z = pack16(__uint_as_float(v[g][4]) * inv, __uint_as_float(v[g][5]) * inv, p.bf16);
+              w0.w = pack16(__uint_as_float(v[g][6]) * inv, __uint_as_float(v[g][7]) * inv, p.bf16);
+              w1.x = pack16(__uint_as_float(v[g][8]) * inv, __uint_as_float(v[g][9]) * inv, p.bf16);
+              w1.y = pack16(__uint_as_float(v[g][10]) * inv, __uint_as_float(v[g][11]) * inv, p.bf16);
+              w1.z = pack16(__uint_as_float(v[g][12]) * inv, __uint_as_float(v[g][13]) * inv, p.bf16);
+              w1.w = pack16(__uint_as_float(v[g][14]) * inv, __uint_as_float(v[g][15]) * inv, p.bf16);
+              *reinterpret_cast<uint4*>(orow + (c0 + g * 16) * 2) = w0;
+              *reinterpret_cast<uint4*>(orow + (c0 + g * 16) * 2 + 16) = w1;
+            }
           }
         }
       }
