@@ -677,7 +677,8 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
             int* splits_out, long long* stride_out, const GemmOpts& o = GemmOpts(), bool* fused_out = nullptr) {
   static PerDeviceOnce attr_once;
   if (attr_once.need()) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+    if (cudaFuncSetAttribute(k_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(k_gemm_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(k_gemm_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return DKV_E_CUDA;
   }
@@ -781,7 +782,8 @@ int gemm_tc(const CUtensorMap& tw, const CUtensorMap* xmaps /*[N_BOX]*/, int n, 
     set_tail(p, o.tail);
     if (fused_out) *fused_out = true;
   }
-  launch_k(k_gemm_tc, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps[bi], p);
+  if (plan.halves == 2) launch_k(k_gemm_tc<2>, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps[bi], p);
+  else launch_k(k_gemm_tc<1>, grid, GEMM_THREADS, plan.smem_bytes, st, tw, xmaps[bi], p);
   *splits_out = splits;
   *stride_out = p.split_stride;
   return cudaGetLastError() == cudaSuccess ? DKV_OK : DKV_E_CUDA;

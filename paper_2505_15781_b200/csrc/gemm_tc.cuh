@@ -334,6 +334,7 @@ __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int 
   return true;
 }
 
+template <int HALVES>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_x, GemmTcParams p) {
   const int STAGES = p.stages;
@@ -350,8 +351,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int a_bytes = p.halves * GEMM_A_BYTES;
-  const int tile_rows = p.halves * GEMM_BM;
+  const int a_bytes = HALVES * GEMM_A_BYTES;
+  const int tile_rows = HALVES * GEMM_BM;
 
   // unit u -> (weight tile, row tile, split); consecutive units differ in the split first
   auto decode = [&](int u, int& n0, int& r0, int& split, int& kb0, int& n_kb) {
@@ -388,7 +389,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const uint32_t full = smem_u32(&bars[s]);
     mbar_expect_tx(full, static_cast<uint32_t>(p.stage_bytes));
     const uint32_t a_dst = smem_base + s * p.stage_bytes;
-    for (int h = 0; h < p.halves; ++h)
+    for (int h = 0; h < HALVES; ++h)
       if (p.w_blocked)      // block (row block, k-block) of a blocked copy: rows block * 128 .. + 127 of its map
         tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, 0,
                          (c.n0 + h * GEMM_BM) * p.kb_total + (c.kb0 + c.i) * GEMM_BM, pol_w);
@@ -474,7 +475,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         ok = mbar_wait_bounded(smem_u32(&acc_empty[buf]), (use & 1) ^ 1, abort_flag, GEMM_WAIT_CYCLES);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * p.halves * p.col_stride);
+        const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * HALVES * p.col_stride);
         for (int i = 0; i < n_kb; ++i, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -483,7 +484,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           tc_fence_after();
           const uint32_t a_addr = smem_base + s * p.stage_bytes;
           const uint64_t bdesc = umma_desc_sw128(a_addr + a_bytes);
-          for (int h = 0; h < p.halves; ++h) {
+          for (int h = 0; h < HALVES; ++h) {
             const uint64_t adesc = umma_desc_sw128(a_addr + h * GEMM_A_BYTES);
 #pragma unroll
             for (int k4 = 0; k4 < GEMM_BK / 16; ++k4) {
@@ -583,10 +584,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
           }
         }
       } else
-      for (int h = 0; h < p.halves; ++h) {
+      for (int h = 0; h < HALVES; ++h) {
         const int n = n0 + h * GEMM_BM + q * 32 + lane;
         const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) +
-                                static_cast<uint32_t>((buf * p.halves + h) * p.col_stride);
+                                static_cast<uint32_t>((buf * HALVES + h) * p.col_stride);
         for (int c = cs * 16; c < p.br; c += 32) {
           if (r0 + c >= r_valid) break;
           uint32_t v[16];
