@@ -384,8 +384,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     }
     return false;
   };
-  auto load_a = [&](const Cursor& c, int it) {
-    const int s = it % STAGES;
+  auto load_a = [&](const Cursor& c, int s) {
     const uint32_t full = smem_u32(&bars[s]);
     mbar_expect_tx(full, static_cast<uint32_t>(p.stage_bytes));
     const uint32_t a_dst = smem_base + s * p.stage_bytes;
@@ -396,8 +395,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
       else
         tma_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, full, (c.kb0 + c.i) * GEMM_BK, c.n0 + h * GEMM_BM, pol_w);
   };
-  auto load_b = [&](const Cursor& c, int it) {
-    const int s = it % STAGES;
+  auto load_b = [&](const Cursor& c, int s) {
     tma_load_2d_hint(smem_base + s * p.stage_bytes + a_bytes, &tm_x, smem_u32(&bars[s]), (c.kb0 + c.i) * GEMM_BK,
                      c.r0, pol_x);
   };
@@ -447,24 +445,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         load_b(c, it);
         ++c.i;
       }
-      int it = pre;
+      // ring position without divisions: stage s, phase bit ph (flips on every wrap)
+      int s = pre == STAGES ? 0 : pre;
+      uint32_t ph = pre == STAGES ? 1u : 0u;
       bool ok = true;
       while (ok && settle(c)) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
         ok = mbar_wait_bounded(smem_u32(&bars[STAGES + s]), ph ^ 1, abort_flag, GEMM_WAIT_CYCLES);
         if (!ok) break;
-        load_a(c, it);
-        load_b(c, it);
+        load_a(c, s);
+        load_b(c, s);
         ++c.i;
-        ++it;
+        if (++s == STAGES) {
+          s = 0;
+          ph ^= 1u;
+        }
       }
     }
   } else if (warp == 1) {
     // --------------------------------------------------------- MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_f16(GEMM_BM, p.br, p.x_bf16);
-      int it = 0, j = 0;
+      int s = 0, j = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++j) {
         int n0, r0, split, kb0, n_kb;
@@ -476,9 +478,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * HALVES * p.col_stride);
-        for (int i = 0; i < n_kb; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int i = 0; i < n_kb; ++i) {
           ok = mbar_wait_bounded(smem_u32(&bars[s]), ph, abort_flag, GEMM_WAIT_CYCLES);
           if (!ok) break;
           tc_fence_after();
@@ -494,6 +494,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             }
           }
           umma_commit(smem_u32(&bars[STAGES + s]));   // frees the smem stage when the MMAs are done
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
         if (ok) umma_commit(smem_u32(&acc_full[buf]));  // accumulator complete (also when n_kb == 0)
       }

@@ -172,8 +172,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         }
         return false;
       };
-      auto load_a = [&](const Cursor& c, int it) {
-        const int s = it % STAGES;
+      auto load_a = [&](const Cursor& c, int s) {
         // the leader announces the bytes of BOTH CTAs' loads of this stage
         if (rank == 0) mbar_expect_tx(smem_u32(&full[s]), static_cast<uint32_t>(2 * (a_bytes + b_bytes)));
         const uint32_t lf = mapa_shared(smem_u32(&full[s]), 0);
@@ -187,8 +186,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
             tma_pair_load_2d_hint(a_dst + h * GEMM_A_BYTES, &tm_w, lf, (c.kb0 + c.i) * GEMM_BK,
                                   c.n0 + static_cast<int>(rank) * 256 + h * GEMM_BM, pol_w);
       };
-      auto load_b = [&](const Cursor& c, int it) {
-        const int s = it % STAGES;
+      auto load_b = [&](const Cursor& c, int s) {
         const uint32_t lf = mapa_shared(smem_u32(&full[s]), 0);
         tma_pair_load_2d_hint(smem_base + s * p.stage_bytes + a_bytes, &tm_x, lf, (c.kb0 + c.i) * GEMM_BK,
                               c.r0 + static_cast<int>(rank) * b_rows, pol_x);
@@ -208,24 +206,28 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         load_b(c, it);
         ++c.i;
       }
-      int it = pre;
+      // ring position without divisions: stage s, phase bit ph (flips on every wrap)
+      int s = pre == STAGES ? 0 : pre;
+      uint32_t ph = pre == STAGES ? 1u : 0u;
       bool ok = true;
       while (ok && settle(c)) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
         ok = mbar_wait_bounded(smem_u32(&empty[s]), ph ^ 1, abort_flag, GEMM_WAIT_CYCLES);
         if (!ok) break;
-        load_a(c, it);
-        load_b(c, it);
+        load_a(c, s);
+        load_b(c, s);
         ++c.i;
-        ++it;
+        if (++s == STAGES) {
+          s = 0;
+          ph ^= 1u;
+        }
       }
     }
   } else if (warp == 1) {
     // --------------------------------------------------------- MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = umma_idesc_f16(256, p.br, p.x_bf16);
-      int it = 0, j = 0;
+      int s = 0, j = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int u = pair; u < p.units && ok; u += n_pairs, ++j) {
         int n0, r0, split, kb0, n_kb;
@@ -236,9 +238,7 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * 2 * p.col_stride);
-        for (int i = 0; i < n_kb; ++i, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int i = 0; i < n_kb; ++i) {
           ok = mbar_wait_bounded(smem_u32(&full[s]), ph, abort_flag, GEMM_WAIT_CYCLES);
           if (!ok) break;
           tc_fence_after();
@@ -252,6 +252,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
                             (i > 0 || k4 > 0) ? 1u : 0u);
           }
           umma_pair_commit(smem_u32(&empty[s]));      // frees the stage in both CTAs
+          if (++s == STAGES) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
         if (ok) umma_pair_commit(smem_u32(&acc_full[buf]));
       }
