@@ -372,15 +372,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
   const uint64_t pol_x = l2_policy_evict_last();    // the few activation rows are re-read by every CTA
   struct Cursor {
     int u, i, n0, r0, split, kb0, n_kb;
+    bool decoded;      // the unit's fields are valid (the divisions of decode() run once per unit, not per k-block)
   } cur, head;
   cur.u = blockIdx.x;
   cur.i = 0;
+  cur.decoded = false;
   auto settle = [&](Cursor& c) {   // move to the next k-block that exists (or past the end)
     while (c.u < p.units) {
-      decode(c.u, c.n0, c.r0, c.split, c.kb0, c.n_kb);
+      if (!c.decoded) {
+        decode(c.u, c.n0, c.r0, c.split, c.kb0, c.n_kb);
+        c.decoded = true;
+      }
       if (c.i < c.n_kb) return true;
       c.u += gridDim.x;
       c.i = 0;
+      c.decoded = false;
     }
     return false;
   };
