@@ -485,21 +485,28 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         tc_fence_after();
         const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * HALVES * p.col_stride);
         for (int i = 0; i < n_kb; ++i) {
-          ok = mbar_wait_bounded(smem_u32(&bars[s]), ph, abort_flag, GEMM_WAIT_CYCLES);
-          if (!ok) break;
-          tc_fence_after();
+          // everything that depends only on the stage is computed BEFORE the wait: what this thread
+          // executes between the arrival of a stage and its MMAs is on the main loop's critical path
           const uint32_t a_addr = smem_base + s * p.stage_bytes;
           const uint64_t bdesc = umma_desc_sw128(a_addr + a_bytes);
+          uint64_t adesc[HALVES];
+#pragma unroll
+          for (int h = 0; h < HALVES; ++h) adesc[h] = umma_desc_sw128(a_addr + h * GEMM_A_BYTES);
+          const uint32_t full_bar = smem_u32(&bars[s]), empty_bar = smem_u32(&bars[STAGES + s]);
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
+          ok = mbar_wait_bounded(full_bar, ph, abort_flag, GEMM_WAIT_CYCLES);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
           for (int h = 0; h < HALVES; ++h) {
-            const uint64_t adesc = umma_desc_sw128(a_addr + h * GEMM_A_BYTES);
 #pragma unroll
             for (int k4 = 0; k4 < GEMM_BK / 16; ++k4) {
               // advance 16 elements = 32 bytes inside the swizzle row: +2 in the (addr >> 4) field
-              umma_f16(d_base + static_cast<uint32_t>(h * p.col_stride), adesc + 2 * k4, bdesc + 2 * k4, idesc,
-                       (i > 0 || k4 > 0) ? 1u : 0u);
+              umma_f16(d_base + static_cast<uint32_t>(h * p.col_stride), adesc[h] + 2 * k4, bdesc + 2 * k4, idesc,
+                       k4 > 0 ? 1u : acc0);
             }
           }
-          umma_commit(smem_u32(&bars[STAGES + s]));   // frees the smem stage when the MMAs are done
+          umma_commit(empty_bar);   // frees the smem stage when the MMAs are done
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;

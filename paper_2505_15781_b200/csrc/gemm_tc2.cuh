@@ -239,19 +239,24 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
         tc_fence_after();
         const uint32_t d_base = tmem_base + static_cast<uint32_t>(buf * 2 * p.col_stride);
         for (int i = 0; i < n_kb; ++i) {
-          ok = mbar_wait_bounded(smem_u32(&full[s]), ph, abort_flag, GEMM_WAIT_CYCLES);
-          if (!ok) break;
-          tc_fence_after();
+          // everything that depends only on the stage is computed BEFORE the wait: what this thread
+          // executes between the arrival of a stage and its MMAs is on the main loop's critical path
           const uint32_t a_addr = smem_base + s * p.stage_bytes;
           const uint64_t bdesc = umma_desc_sw128(a_addr + a_bytes);
-          for (int h = 0; h < 2; ++h) {
-            const uint64_t adesc = umma_desc_sw128(a_addr + h * GEMM_A_BYTES);
+          const uint64_t adesc0 = umma_desc_sw128(a_addr), adesc1 = umma_desc_sw128(a_addr + GEMM_A_BYTES);
+          const uint32_t full_bar = smem_u32(&full[s]), empty_bar = smem_u32(&empty[s]);
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
+          ok = mbar_wait_bounded(full_bar, ph, abort_flag, GEMM_WAIT_CYCLES);
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
-            for (int k4 = 0; k4 < GEMM_BK / 16; ++k4)
-              umma_pair_f16(d_base + static_cast<uint32_t>(h * p.col_stride), adesc + 2 * k4, bdesc + 2 * k4, idesc,
-                            (i > 0 || k4 > 0) ? 1u : 0u);
-          }
-          umma_pair_commit(smem_u32(&empty[s]));      // frees the stage in both CTAs
+          for (int k4 = 0; k4 < GEMM_BK / 16; ++k4)
+            umma_pair_f16(d_base, adesc0 + 2 * k4, bdesc + 2 * k4, idesc, k4 > 0 ? 1u : acc0);
+#pragma unroll
+          for (int k4 = 0; k4 < GEMM_BK / 16; ++k4)
+            umma_pair_f16(d_base + static_cast<uint32_t>(p.col_stride), adesc1 + 2 * k4, bdesc + 2 * k4, idesc,
+                          k4 > 0 ? 1u : acc0);
+          umma_pair_commit(empty_bar);      // frees the stage in both CTAs
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
