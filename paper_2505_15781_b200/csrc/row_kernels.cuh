@@ -34,24 +34,7 @@ __device__ __forceinline__ float block_sum_256(float v, float* s8) {
   return t;
 }
 
-// fp16 copy of a bf16 matrix (values below 2^-14 lose bits: |error| <= 2^-25)
-__global__ void __launch_bounds__(256) k_bf16_to_f16(const __nv_bfloat16* __restrict__ in, __half* __restrict__ out,
-                                                      size_t n) {
-  const size_t n8 = n / 8;
-  for (size_t i = blockIdx.x * 256ull + threadIdx.x; i < n8; i += gridDim.x * 256ull) {
-    const uint4 v = reinterpret_cast<const uint4*>(in)[i];
-    const __nv_bfloat162* b = reinterpret_cast<const __nv_bfloat162*>(&v);
-    uint4 o;
-    __half2* h = reinterpret_cast<__half2*>(&o);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) h[j] = __float22half2_rn(__bfloat1622float2(b[j]));
-    reinterpret_cast<uint4*>(out)[i] = o;
-  }
-  for (size_t i = n8 * 8 + blockIdx.x * 256ull + threadIdx.x; i < n; i += gridDim.x * 256ull)
-    out[i] = __float2half_rn(__bfloat162float(in[i]));
-}
-
-// fp16 copy of a bf16 weight matrix [rows, k] in blocks of 128 rows x 64 columns, block (i, j) at
+// fp16 copy of a bf16 weight matrix [rows, k] (values below 2^-14 lose bits: |error| <= 2^-25) in blocks of 128 rows x 64 columns, block (i, j) at
 // (i * ceil(k / 64) + j) * 8192 elements, rows inside a block 64 elements apart, zeros past the
 // matrix: what the projection GEMM loads per weight half and k-block is one contiguous 16 KB piece.
 // With gu_blk > 0 the matrix is [gate (gu_f rows); up (gu_f rows)] and the copy's rows are regrouped
