@@ -528,7 +528,7 @@ void choose_multi_tile(int n, int k, int r_bound, long long part_rows, int* tile
 
 // The same estimate for a launch on CTA pairs (k_gemm_tc2): a unit is 512 weight rows x br rows on two
 // SMs, each CTA takes in 32 KB of weights and br / 2 rows per k-block, and the units run in waves of
-// NUM_SMS / 2 pairs.  `one_wave`: only plans whose units are all resident at once (fused row tails).
+// NUM_SMS / 2 pairs.
 double est_clocks_pairs(int n, int k, int r_bound, int t, int s) {
   const int per = ceil_div(r_bound, t);
   const int br = 16 * ceil_div(per, 16);
@@ -541,6 +541,8 @@ double est_clocks_pairs(int n, int k, int r_bound, int t, int s) {
   const double partials = s > 1 ? 4.0 * s * r_bound * static_cast<double>(n) / (4.0e12 / 1.85e9) : 0.0;
   return waves * unit + partials;
 }
+// Row tiles and K splits of a pair launch; `one_wave`: only plans whose units are all resident at once
+// (what the fused row tails need).  Zero tiles: no such plan.
 double choose_pairs(int n, int k, int r_bound, long long part_rows, bool one_wave, int* tiles_out, int* splits_out) {
   const int kb_total = ceil_div(k, GEMM_BK);
   int s_max = std::min(8, std::max(1, kb_total / 4));
