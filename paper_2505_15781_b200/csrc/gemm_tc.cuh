@@ -439,7 +439,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const unsigned long long t_enter = (trace_on() && threadIdx.x == 64) ? global_timer_ns() : 0ull;
+  // (only the one recording thread looks at the trace switch, a word in global memory: the single-thread
+  // roles must not wait for that load)
+  const unsigned long long t_enter = (threadIdx.x == 64 && trace_on()) ? global_timer_ns() : 0ull;
 
   if (warp == 0) {
     // ------------------------------------------------------- TMA producer
@@ -522,7 +524,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const int et = threadIdx.x - 64;  // 0..255 among the epilogue threads
     float* s_rs = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + GEMM_BAR_BYTES);   // [256] row scales
     pdl_wait();              // the row count and the output buffer belong to earlier kernels
-    if (trace_on() && threadIdx.x == 64) trace_store(3, t_enter);
+    if (threadIdx.x == 64 && trace_on()) trace_store(3, t_enter);
     int r_valid = p.r_bound;
     if (p.r_dev) r_valid = min(r_valid, *p.r_dev);
     // head mode: the statistics of this warp's token ids over ALL weight tiles of the CTA, per row

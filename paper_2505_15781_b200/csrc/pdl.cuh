@@ -44,7 +44,7 @@ __device__ __forceinline__ void trace_store(int kernel_id, unsigned long long t_
 
 // the common case: nothing useful to do before the predecessor's data is ready
 __device__ __forceinline__ void pdl_enter(int kernel_id = 0) {
-  const bool tr = trace_on() && threadIdx.x == 0;
+  const bool tr = threadIdx.x == 0 && trace_on();   // (one thread reads the switch, a word in global memory)
   const unsigned long long t0 = tr ? global_timer_ns() : 0ull;
   pdl_launch();
   pdl_wait();
