@@ -212,8 +212,10 @@ __device__ __forceinline__ void sum_splits(const GemmTcParams& p, const long lon
   }
 }
 
+// (`g`: the lane's gains, loaded by the caller before the wait for the tile's splits — nothing that does
+// not depend on the sums may add a round trip through L2 after them)
 __device__ __forceinline__ void fused_rows_resid(const GemmTcParams& p, int n0, int tile_rows, int row_lo, int row_hi,
-                                                 int ewarp, int lane) {
+                                                 int ewarp, int lane, const float4 (&g)[2]) {
   const int tile_n = n0 / tile_rows;
   for (int rb = row_lo + ewarp * FUSE_ROWS; rb < row_hi; rb += 8 * FUSE_ROWS) {
     long long at[FUSE_ROWS * 2];
@@ -237,9 +239,8 @@ __device__ __forceinline__ void fused_rows_resid(const GemmTcParams& p, int n0, 
           const float4 a = acc[i];
           *reinterpret_cast<float4*>(p.h + at[i]) = a;
           ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
-          const float4 g = __ldg(reinterpret_cast<const float4*>(p.gain + n0 + hf * 128 + lane * 4));
           *reinterpret_cast<uint2*>(static_cast<uint16_t*>(p.xn_out) + at[i]) =
-              pack4_16(a.x * g.x, a.y * g.y, a.z * g.z, a.w * g.w, p.x_bf16);
+              pack4_16(a.x * g[hf].x, a.y * g[hf].y, a.z * g[hf].z, a.w * g[hf].w, p.x_bf16);
         }
       }
 #pragma unroll
@@ -251,8 +252,12 @@ __device__ __forceinline__ void fused_rows_resid(const GemmTcParams& p, int n0, 
 
 // A tile of 256 columns holds 256 / head_dim whole heads and a head's rotation pairs are (i, i + head_dim/2):
 // head_dim / 8 lanes per head, each with pairs i..i+3, is exactly one warp per row (head_dim 64 or 128).
+// `flat0`: the flattened positions of the warp's first FUSE_ROWS rows, loaded by the caller before the
+// wait for the tile's splits; the positions of the next pass are requested while this pass runs, and
+// a pass asks for its rotation factors BEFORE its partial sums: neither the position nor the table
+// entry may add a round trip through L2 after the sums.
 __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, int tile_rows, int row_lo, int row_hi,
-                                               int ewarp, int lane) {
+                                               int ewarp, int lane, const int (&flat0)[FUSE_ROWS]) {
   const int hd = p.head_dim, half = hd >> 1;
   const int lanes_per_head = hd >> 3;
   const int hh = lane / lanes_per_head, i0 = (lane - hh * lanes_per_head) * 4;
@@ -263,10 +268,29 @@ __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, in
   const bool is_q = head < p.n_q_heads;
   const bool rot = head < p.n_q_heads + p.n_kv_heads;
   const int hk = head - p.n_q_heads - (rot ? 0 : p.n_kv_heads);
+  int flat_next[FUSE_ROWS];
+#pragma unroll
+  for (int rr = 0; rr < FUSE_ROWS; ++rr) flat_next[rr] = flat0[rr];
   for (int rb = row_lo + ewarp * FUSE_ROWS; rb < row_hi; rb += 8 * FUSE_ROWS) {
     long long at[FUSE_ROWS * 2];
     bool on[FUSE_ROWS * 2];
     float4 acc[FUSE_ROWS * 2];
+    int bq[FUSE_ROWS], posq[FUSE_ROWS];
+    float4 t0q[FUSE_ROWS], t1q[FUSE_ROWS];
+#pragma unroll
+    for (int rr = 0; rr < FUSE_ROWS; ++rr) {
+      const int flat = flat_next[rr];
+      const int rn = rb + 8 * FUSE_ROWS + rr;                  // the same warp's row of the next pass
+      flat_next[rr] = rn < row_hi ? p.act_idx[rn] : 0;
+      bq[rr] = flat / p.seq_len;
+      posq[rr] = flat - bq[rr] * p.seq_len;
+      t0q[rr] = t1q[rr] = make_float4(1.f, 0.f, 1.f, 0.f);
+      if (rot && head_on && rb + rr < row_hi) {
+        const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + static_cast<long long>(posq[rr]) * half + i0);
+        t0q[rr] = __ldg(tab);                                  // (cos, sin) of i0, i0+1
+        t1q[rr] = __ldg(tab + 1);                              // (cos, sin) of i0+2, i0+3
+      }
+    }
 #pragma unroll
     for (int i = 0; i < FUSE_ROWS * 2; ++i) {
       const int r = rb + (i >> 1);
@@ -279,12 +303,10 @@ __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, in
     for (int rr = 0; rr < FUSE_ROWS; ++rr) {
       const int r = rb + rr;
       if (!on[rr * 2]) continue;
-      const int flat = p.act_idx[r];
-      const int b = flat / p.seq_len, pos = flat - b * p.seq_len;
+      const int b = bq[rr], pos = posq[rr];
       float4 x1 = acc[rr * 2], x2 = acc[rr * 2 + 1];
       if (rot) {
-        const float4* tab = reinterpret_cast<const float4*>(p.rope_tab + static_cast<long long>(pos) * half + i0);
-        const float4 t0 = __ldg(tab), t1 = __ldg(tab + 1);      // (cos, sin) of i0, i0+1 | i0+2, i0+3
+        const float4 t0 = t0q[rr], t1 = t1q[rr];
         const float4 y1 = make_float4(x1.x * t0.x - x2.x * t0.y, x1.y * t0.z - x2.y * t0.w,
                                       x1.z * t1.x - x2.z * t1.y, x1.w * t1.z - x2.w * t1.w);
         const float4 y2 = make_float4(x2.x * t0.x + x1.x * t0.y, x2.y * t0.z + x1.y * t0.w,
@@ -309,6 +331,25 @@ __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, in
 __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int split, int n0, int tile_rows, int r0,
                                            int r_valid, volatile int* abort_flag, int et, int ewarp, int lane) {
   unsigned int* cnt = p.tile_cnt + tile;
+  // this CTA's share of the tile's rows, and what its warps need beside the sums (gains; the first
+  // rows' positions), requested before the wait
+  const int n_rows = max(0, min(p.br, r_valid - r0));
+  const int per = (n_rows + p.splits - 1) / p.splits;
+  const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
+  float4 gains[2];
+  int flat0[FUSE_ROWS];
+#pragma unroll
+  for (int hf = 0; hf < 2; ++hf) {
+    const int n = n0 + hf * 128 + lane * 4;
+    gains[hf] = (p.fuse_mode == FUSE_RESID && hf * 128 < tile_rows && n < p.n)
+                    ? __ldg(reinterpret_cast<const float4*>(p.gain + n))
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int rr = 0; rr < FUSE_ROWS; ++rr) {
+    const int r = row_lo + ewarp * FUSE_ROWS + rr;
+    flat0[rr] = (p.fuse_mode == FUSE_QKV && r < row_hi) ? p.act_idx[r] : 0;
+  }
   __threadfence();
   named_bar_sync(2, 256);
   bool fail = false;
@@ -326,11 +367,8 @@ __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int 
     __threadfence();
   }
   if (bar_red_or(2, 256, fail)) return false;
-  const int n_rows = max(0, min(p.br, r_valid - r0));
-  const int per = (n_rows + p.splits - 1) / p.splits;
-  const int row_lo = r0 + min(n_rows, split * per), row_hi = r0 + min(n_rows, (split + 1) * per);
-  if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, ewarp, lane);
-  else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, ewarp, lane);
+  if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, gains);
+  else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, flat0);
   return true;
 }
 
