@@ -363,12 +363,15 @@ __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int 
         break;
       }
     }
-    if (!fail && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;   // everyone has passed: reset
-    __threadfence();
   }
+  // (thread 0's acquire and the barrier order the other splits' sums before every thread's loads)
   if (bar_red_or(2, 256, fail)) return false;
   if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, gains);
   else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, flat0);
+  // Past the wait: counted a second time, and the last CTA of the tile to get here resets the counter
+  // for the next launch.  After the row work, not before it: the answer of this atomic is a round trip
+  // through L2 that nothing of the tail needs.
+  if (et == 0 && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;
   return true;
 }
 
