@@ -282,7 +282,7 @@ struct Arena {
   float* part;
   float* ssq;                    // [ceil(d_model / 128)][r_cap]: partial sums of squares of the residual rows
   float* head_rs;                // [h_cap]: 1 / RMS of each head row
-  unsigned int* tile_cnt;        // [MAX_TILE_COUNTERS]: arrival counters of the fused GEMM tails
+  unsigned int* tile_cnt;        // [2][MAX_TILE_COUNTERS]: arrival counters of the fused GEMM tails, two sets used in turn
   float* conf_i;
   int32_t* pred_i;
   int32_t* tok_stage;
@@ -359,7 +359,7 @@ void carve(const dkv_model* m, const Dims& d, uint8_t* base, Arena* a) {
   a->part = reinterpret_cast<float*>(take(d.part_rows * d.n_max * 4));
   a->ssq = reinterpret_cast<float*>(take(static_cast<size_t>((md.d_model + 127) / 128) * d.r_cap * 4));
   a->head_rs = reinterpret_cast<float*>(take(d.h_cap * 4));
-  a->tile_cnt = reinterpret_cast<unsigned int*>(take(MAX_TILE_COUNTERS * 4));
+  a->tile_cnt = reinterpret_cast<unsigned int*>(take(2 * MAX_TILE_COUNTERS * 4));
   a->conf_i = reinterpret_cast<float*>(take(BL * 4));
   a->pred_i = reinterpret_cast<int32_t*>(take(BL * 4));
   a->tok_stage = reinterpret_cast<int32_t*>(take(BL * 4));
@@ -391,6 +391,7 @@ struct dkv_cache {
                          // the O and down GEMMs (one-wave launches)
   long long tail_wait_cycles;   // bound of the fused tails' cross-CTA wait; dkv_debug_tail_wait shortens it
   int tail_extra;               // arrivals the tails expect beyond the real ones (0; 1 under dkv_debug_tail_wait)
+  int tail_cnt_set;             // which of the two sets of tile counters the next fused launch uses
   int step;              // steps run so far
   int last_refresh;      // step number of the last full / generation-only step
   int pending_refresh;   // -1 none, else DKV_REFRESH_*
@@ -620,7 +621,8 @@ struct RowScale {
 // Row epilogue fused into the GEMM across the CTAs of a weight tile (FUSE_RESID / FUSE_QKV).
 struct FusedTail {
   int mode = FUSE_NONE;
-  unsigned int* tile_cnt = nullptr;
+  unsigned int* tile_cnt = nullptr;   // [2][MAX_TILE_COUNTERS]
+  int* cnt_set = nullptr;             // which set the next fused launch counts on (flipped by every fused launch)
   long long wait_cycles = GEMM_WAIT_CYCLES;
   int extra = 0;
   float* h = nullptr;
@@ -651,7 +653,9 @@ struct GemmOpts {
 
 void set_tail(GemmTcParams& p, const FusedTail& t) {
   p.fuse_mode = t.mode;
-  p.tile_cnt = t.tile_cnt;
+  p.tile_cnt = t.tile_cnt + *t.cnt_set * MAX_TILE_COUNTERS;
+  p.tile_cnt_next = t.tile_cnt + (1 - *t.cnt_set) * MAX_TILE_COUNTERS;
+  *t.cnt_set ^= 1;
   p.tail_wait_cycles = t.wait_cycles;
   p.tail_extra = t.extra;
   p.h = t.h;
@@ -916,6 +920,7 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     if (c->fuse_tails & 2) {
       o.tail.mode = FUSE_RESID;
       o.tail.tile_cnt = a.tile_cnt;
+      o.tail.cnt_set = &c->tail_cnt_set;
       o.tail.wait_cycles = c->tail_wait_cycles;
       o.tail.extra = c->tail_extra;
       o.tail.h = a.h;
@@ -969,6 +974,7 @@ int run_forward(dkv_cache* c, const StepPlan& plan, const int32_t* tokens, float
     if ((c->fuse_tails & 1) && R <= 256) {
       o.tail.mode = FUSE_QKV;
       o.tail.tile_cnt = a.tile_cnt;
+      o.tail.cnt_set = &c->tail_cnt_set;
       o.tail.wait_cycles = c->tail_wait_cycles;
       o.tail.extra = c->tail_extra;
       o.tail.act_idx = a.act_idx;
@@ -1456,7 +1462,7 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   }
   const size_t BL = static_cast<size_t>(batch) * seq_len;
   cudaMemsetAsync(a.status, 0, 256, st);
-  cudaMemsetAsync(a.tile_cnt, 0, MAX_TILE_COUNTERS * 4, st);
+  cudaMemsetAsync(a.tile_cnt, 0, 2 * MAX_TILE_COUNTERS * 4, st);
   cudaMemsetAsync(a.written_step, 0, BL * 4, st);
   cudaMemsetAsync(a.mask_buf[0], 0, BL, st);
   cudaMemsetAsync(a.mask_buf[1], 0, BL, st);
@@ -1480,6 +1486,7 @@ int dkv_init_cache(const dkv_model* m, int batch, int seq_len, int prompt_len, c
   c->fuse_tails = env_int("DKV_FUSE_TAILS", 3);
   c->tail_wait_cycles = GEMM_WAIT_CYCLES;
   c->tail_extra = 0;
+  c->tail_cnt_set = 0;
   c->step = 0;
   c->last_refresh = 1;
   c->pending_refresh = -1;

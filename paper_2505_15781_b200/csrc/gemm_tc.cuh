@@ -133,7 +133,9 @@ struct GemmTcParams {
   float rs_inv_d, rs_eps;
   // fused row epilogue across the CTAs of a weight tile (FUSE_*); needs units <= resident CTAs
   int fuse_mode;
-  unsigned int* tile_cnt;  // [weight tiles * row tiles] arrival counters, zero between launches
+  unsigned int* tile_cnt;  // this launch's arrival counters, one per (weight tile, row tile): all zero at its start
+  unsigned int* tile_cnt_next;   // the other set of counters (256): the previous fused launch's, zeroed by this
+                                 // launch for the next one, so that no counter has to be reset behind a wait
   long long tail_wait_cycles;  // bound of the wait for the tile's other CTAs (GEMM_WAIT_CYCLES unless a test shortens it)
   int tail_extra;          // arrivals expected beyond the tile's K splits: 0; a test of the error path sets 1,
                            // so that the wait can only run out
@@ -326,8 +328,9 @@ __device__ __forceinline__ void fused_rows_qkv(const GemmTcParams& p, int n0, in
 // Cross-CTA hand-over of the fused row epilogues, run by the 256 epilogue threads of a CTA after its
 // partial sums of the unit are in scratch: the CTA counts itself on the tile's counter and waits
 // (bounded) until all K splits of the tile are there; then it finishes its own slice of the tile's
-// rows.  `tile` indexes the counters; the tile's columns are [n0, n0 + tile_rows).  The last CTA to
-// get past the wait resets the counter.  Returns false when a wait ran out (the abort flag is set).
+// rows.  `tile` indexes the counters; the tile's columns are [n0, n0 + tile_rows).  The counters are
+// not reset here: fused launches alternate between two sets, and each zeroes the other set once its
+// predecessors have completed.  Returns false when a wait ran out (the abort flag is set).
 __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int split, int n0, int tile_rows, int r0,
                                            int r_valid, volatile int* abort_flag, int et, int ewarp, int lane) {
   unsigned int* cnt = p.tile_cnt + tile;
@@ -368,10 +371,6 @@ __device__ __forceinline__ bool fused_tail(const GemmTcParams& p, int tile, int 
   if (bar_red_or(2, 256, fail)) return false;
   if (p.fuse_mode == FUSE_RESID) fused_rows_resid(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, gains);
   else fused_rows_qkv(p, n0, tile_rows, row_lo, row_hi, ewarp, lane, flat0);
-  // Past the wait: counted a second time, and the last CTA of the tile to get here resets the counter
-  // for the next launch.  After the row work, not before it: the answer of this atomic is a round trip
-  // through L2 that nothing of the tail needs.
-  if (et == 0 && atomicAdd(cnt, 1u) == 2u * p.splits - 1u) *cnt = 0u;
   return true;
 }
 
@@ -565,6 +564,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     const int et = threadIdx.x - 64;  // 0..255 among the epilogue threads
     float* s_rs = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + GEMM_BAR_BYTES);   // [256] row scales
     pdl_wait();              // the row count and the output buffer belong to earlier kernels
+    // (every earlier launch has completed: the counters of the previous fused launch are free to be
+    // zeroed for the next one)
+    if (p.fuse_mode != FUSE_NONE && et == 255)
+      for (int i = blockIdx.x; i < 256; i += gridDim.x) p.tile_cnt_next[i] = 0u;
     if (threadIdx.x == 64 && trace_on()) trace_store(3, t_enter);
     int r_valid = p.r_bound;
     if (p.r_dev) r_valid = min(r_valid, *p.r_dev);

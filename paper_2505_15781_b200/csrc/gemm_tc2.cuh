@@ -272,6 +272,10 @@ k_gemm_tc2(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUt
     const int et = threadIdx.x - 64;  // 0..255 among the epilogue threads
     float* s_rs = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + GEMM_BAR_BYTES);   // [256] row scales
     pdl_wait();
+    // (every earlier launch has completed: the counters of the previous fused launch are free to be
+    // zeroed for the next one)
+    if (p.fuse_mode != FUSE_NONE && et == 255)
+      for (int i = blockIdx.x; i < 256; i += gridDim.x) p.tile_cnt_next[i] = 0u;
     int r_valid = p.r_bound;
     if (p.r_dev) r_valid = min(r_valid, *p.r_dev);
     int j = 0;
