@@ -154,7 +154,7 @@ const char* dkv_strerror(int status);
  * and head matrices are first copied to fp16 into `arena` (caller-owned
  * device memory, 256-byte aligned, at least dkv_model_bytes(desc) bytes, kept
  * alive until dkv_model_destroy): tcgen05 MMAs need both operands in one
- * 16-bit format.  (The copies of the layers' matrices are laid out in blocks
+ * 16-bit format.  (The copies of the layers' matrices and of the head are laid out in blocks
  * of 128 rows x 64 columns, zero-padded; the size includes the padding.)  The copy is exact for |w| >= 2^-14 and within 2^-25
  * absolute below; afterwards only embed and the norm gains of the caller's
  * weights are still read.  In the other modes arena may be NULL and the
